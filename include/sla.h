@@ -1,0 +1,181 @@
+/*
+ * sla.h -- C interface of libsla: span-search and span-attention of N=2 Superlinear attention
+ *          on NVIDIA B200 (sm_100a).
+ *
+ * The library computes, for every query position i of a causal sequence:
+ *
+ *   span-search     (paper: Section "Span search", both equations; Algorithm 1, lines
+ *                    "T <- Anchors(i) \ W", "s_t <- <Q_s(i), K_a(t)>", "TopK")
+ *       anchors  t_s = i + 1 - (s+1)^2,  s = 0 .. n(i)-1,  n(i) = floor(sqrt(i+1))
+ *                (Section "Span attention": anchors at i-(s+1)^{1/p}+1 with p = 1/2)
+ *       score    s_{i,t} = search_scale * <Q_s[i], K[t]>          (K_a = K)
+ *       select   the top_k anchors with the largest score
+ *
+ *   span-attention  (paper: Section "Span attention", equation for A_{i,t}; Algorithm 1, lines
+ *                    "S_t <- [max(0,t-b l(i)), min(i,t+f l(i))]" and "Attention(Q(i),K[J_t],V[J_t])")
+ *       span     S_t = [max(0, t - b*l), min(i, t + f*l)]   closed interval of key positions,
+ *                l = span_len if span_len > 0, else ceil(sqrt(i))
+ *       output   softmax(softmax_scale * <Q[i], K[j]>) . V over j in the union of the selected
+ *                spans (each key counted once), plus lse = log sum_j exp(softmax_scale*<Q[i],K[j]>)
+ *
+ *   decode step     (paper: Section "Kernel design", paragraph "Decoding path")
+ *       the two steps above for the single query i = n_ctx - 1 against a KV cache.
+ *
+ * Conventions fixed by this library where the paper leaves a choice:
+ *   - every anchor with t_s >= 0 is a candidate; ties in the selection go to the smaller s;
+ *   - selected anchors are reported by descending score; when fewer than top_k candidates
+ *     exist the tail is padded with anchor = -1, score = -inf;
+ *   - with grouped-query heads each query head routes on its own against the key head of its
+ *     group (kv head = q head / (n_q_heads / n_kv_heads));
+ *   - no positional encoding and no padding mask are applied.
+ *
+ * Memory: unless a parameter says "host", every tensor pointer is DEVICE memory owned by the
+ * caller, on the device the handle was created for.  The innermost (head_dim) axis is contiguous;
+ * the other strides are given in ELEMENTS.  Base pointers must be 16-byte aligned and every stride
+ * a multiple of 8 elements.  Calls are asynchronous: work is enqueued on the given CUDA stream
+ * (a cudaStream_t passed as void*; NULL = the default stream) and outputs are valid once the stream
+ * reaches that point.  The library allocates device memory only in sla_create (the workspace);
+ * no call allocates per invocation.  One handle must not be used by two streams at the same time
+ * (the workspace is shared).
+ *
+ * Errors: every call returns an sla_status_t; 0 is success, negative values are errors.  When
+ * argument validation fails nothing is launched.  No exception or abort crosses this interface.
+ * Device-side problems (an anchor outside [0, i] handed to sla_span_attention, an internal bounded
+ * wait that ran out) never trap: the kernel records a status word, skips the offending work and
+ * returns; sla_poll_status reports it.
+ */
+#ifndef SLA_H_
+#define SLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SLA_OK = 0,
+    SLA_ERR_INVALID_ARG = -1,    /* NULL pointer, bad shape/stride/alignment, out-of-range value   */
+    SLA_ERR_UNSUPPORTED = -2,    /* valid request that this build does not implement              */
+    SLA_ERR_WORKSPACE = -3,      /* the handle's workspace is too small for this call             */
+    SLA_ERR_CUDA = -4,           /* a CUDA runtime call failed (see sla_last_error)               */
+    SLA_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait expired                            */
+    SLA_ERR_DEVICE_INDEX = -6    /* a kernel met an anchor outside [0, i] and skipped it          */
+} sla_status_t;
+
+typedef enum { SLA_F32 = 0, SLA_BF16 = 1 } sla_dtype_t;
+
+/* SLA_UNION: one softmax over the de-duplicated union of the selected spans (reduces to dense
+ * causal attention when the selection covers every key).  SLA_PER_SPAN (Algorithm 1 literally: one
+ * softmax per span, then the softmax gate of Section "Combination") is not implemented yet and
+ * returns SLA_ERR_UNSUPPORTED. */
+typedef enum { SLA_UNION = 0, SLA_PER_SPAN = 1 } sla_mode_t;
+
+typedef struct sla_handle_s *sla_handle_t; /* opaque; owns the device workspace */
+
+/* Shapes and strides shared by the tensors of one call.
+ *   q_s, q, out : [batch, n_q_heads, Lq, head_dim]      strides q_stride_{b,h,t}, head_dim contiguous
+ *   k, v        : [batch, n_kv_heads, Lkv.., head_dim]  strides kv_stride_{b,h,t}
+ * For sla_decode_step the query tensors are [batch, n_q_heads, head_dim] and q_stride_t is ignored. */
+typedef struct {
+    int32_t batch, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0, group size <= 16        */
+    int32_t head_dim;                     /* 64 or 128                                             */
+    int32_t dtype;                        /* sla_dtype_t of q_s, q, k, v and out                   */
+    int32_t reserved;                     /* must be 0                                             */
+    int64_t q_stride_b, q_stride_h, q_stride_t;
+    int64_t kv_stride_b, kv_stride_h, kv_stride_t;
+} sla_layout_t;
+
+typedef struct {
+    int32_t top_k;        /* 1 .. 64                                                              */
+    int32_t span_len;     /* l > 0: fixed base span length; 0: l(i) = ceil(sqrt(i)) (Algorithm 1)  */
+    int32_t back_factor;  /* b >= 0; b >= 2 is needed for full coverage (Section "Span attention") */
+    int32_t fwd_factor;   /* f >= 0                                                               */
+    int32_t window;       /* local window w of Algorithm 1; only 0 is implemented                 */
+    int32_t mode;         /* sla_mode_t; only SLA_UNION is implemented                            */
+    float search_scale;   /* multiplies the search score (the paper's equation has none: 1.0f)    */
+    float softmax_scale;  /* multiplies the attention logits ("scaled dot-product": 1/sqrt(D))     */
+} sla_params_t;
+
+/* ---- handle ------------------------------------------------------------------------------- */
+
+/* Creates a handle on CUDA device `device` and allocates `workspace_bytes` of device scratch memory
+ * (the only allocation the library ever makes; ask sla_workspace_bytes for the size).  The handle
+ * and its workspace are released by sla_destroy.  *handle is set to NULL on failure. */
+sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes);
+sla_status_t sla_destroy(sla_handle_t handle);
+
+/* Scratch bytes that sla_span_search + sla_span_attention with Lq query rows against Lkv keys, and
+ * sla_decode_step at n_ctx = Lkv, need for this layout and these parameters.  Returns 0 when the
+ * arguments are invalid.  Host-only: touches no device. */
+size_t sla_workspace_bytes(const sla_layout_t *layout, const sla_params_t *params, int64_t Lq,
+                           int64_t Lkv);
+
+const char *sla_status_string(sla_status_t status); /* static string, never NULL                  */
+const char *sla_last_error(sla_handle_t handle);    /* text of the last failure on this handle     */
+
+/* Waits for `stream` and reads the device status word: SLA_OK, SLA_ERR_DEVICE_TIMEOUT or
+ * SLA_ERR_DEVICE_INDEX; the word is cleared. */
+sla_status_t sla_poll_status(sla_handle_t handle, void *stream);
+
+/* ---- span-search (Section "Span search"; Algorithm 1 scoring and TopK lines) -------------- */
+
+/* Query row r (0 <= r < Lq) is position i = q_pos0 + r; keys 0 .. Lkv-1 are valid; requires
+ * q_pos0 + Lq <= Lkv.  Full prefill: q_pos0 = 0, Lq = Lkv = L.  A chunk of a chunked prefill:
+ * q_pos0 = first position of the chunk.
+ *   q_s        in   [B, Hq, Lq, D]  device
+ *   k          in   [B, Hkv, >=Lkv, D]  device
+ *   out_anchor out  [B, Hq, Lq, top_k] int32, contiguous, device: key positions, best first, -1 pad
+ *   out_score  out  [B, Hq, Lq, top_k] fp32,  contiguous, device: matching scores, -inf pad        */
+sla_status_t sla_span_search(sla_handle_t handle, const void *q_s, const void *k, int64_t Lq,
+                             int64_t q_pos0, int64_t Lkv, const sla_layout_t *layout,
+                             const sla_params_t *params, int32_t *out_anchor, float *out_score,
+                             void *stream);
+
+/* ---- span-attention (Section "Span attention", equation for A_{i,t}; Algorithm 1 span lines) */
+
+/* The anchors may come from any router; entries < 0 are ignored, entries > i are skipped and
+ * flagged (SLA_ERR_DEVICE_INDEX on the next sla_poll_status).  Overlapping spans of one row are
+ * attended once.
+ *   q          in   [B, Hq, Lq, D] device;  k, v in [B, Hkv, >=Lkv, D] device
+ *   anchor     in   [B, Hq, Lq, top_k] int32, contiguous, device
+ *   out        out  [B, Hq, Lq, D] in the input dtype, strides as q, device
+ *   lse        out  [B, Hq, Lq] fp32, contiguous, device; natural log of the softmax denominator;
+ *                   -inf (and out = 0) for a row with no valid anchor                              */
+sla_status_t sla_span_attention(sla_handle_t handle, const void *q, const void *k, const void *v,
+                                int64_t Lq, int64_t q_pos0, int64_t Lkv, const sla_layout_t *layout,
+                                const sla_params_t *params, const int32_t *anchor, void *out,
+                                float *lse, void *stream);
+
+/* ---- decode step (Section "Kernel design", "Decoding path") -------------------------------- */
+
+/* One new token per sequence.  The caller has already appended the token's key and value to the
+ * cache: positions 0 .. n_ctx-1 are valid and the query position is i = n_ctx - 1.
+ *   q_s, q     in   [B, Hq, D] device (strides q_stride_b, q_stride_h)
+ *   k_cache, v_cache in [B, Hkv, capacity >= n_ctx, D] device (kv strides)
+ *   out        out  [B, Hq, D] input dtype, strides as q;  lse out [B, Hq] fp32 contiguous
+ *   out_anchor out  [B, Hq, top_k] int32 contiguous; out_score out [B, Hq, top_k] fp32 contiguous  */
+sla_status_t sla_decode_step(sla_handle_t handle, const void *q_s, const void *q, const void *k_cache,
+                             const void *v_cache, int64_t n_ctx, const sla_layout_t *layout,
+                             const sla_params_t *params, void *out, float *lse, int32_t *out_anchor,
+                             float *out_score, void *stream);
+
+/* ---- host-buffer convenience calls ---------------------------------------------------------- */
+
+/* sla_span_search followed by sla_span_attention on HOST buffers (pinned memory gives the best
+ * copy rate): copies q_s, q, k, v to the device, runs both steps, copies out, lse, anchors and
+ * scores back, and waits for completion.  All tensors are dense and contiguous
+ * ([B,Hq,L,D] / [B,Hkv,L,D], q_pos0 = 0, Lq = Lkv = L); the layout's strides are ignored.  The
+ * device staging buffers come out of the handle's workspace, which therefore has to be
+ * sla_workspace_bytes(...) + sla_host_staging_bytes(...) large.  Section references as above. */
+size_t sla_host_staging_bytes(const sla_layout_t *layout, const sla_params_t *params, int64_t L);
+sla_status_t sla_prefill_host(sla_handle_t handle, const void *q_s_host, const void *q_host,
+                              const void *k_host, const void *v_host, int64_t L,
+                              const sla_layout_t *layout, const sla_params_t *params, void *out_host,
+                              float *lse_host, int32_t *anchor_host, float *score_host, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLA_H_ */

@@ -1,0 +1,274 @@
+// Host side of libsla: handle, argument validation, workspace carving and kernel dispatch.
+// Every exported function is declared and documented in include/sla.h.
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "sla_kernels.h"
+
+struct sla_handle_s {
+    int device = 0;
+    int sm_count = 0;
+    char *ws = nullptr;       // device workspace; the first kHeaderBytes hold the status word
+    size_t ws_bytes = 0;
+    char err[256] = {0};
+};
+
+namespace {
+
+constexpr size_t kHeaderBytes = 256;
+
+sla_status_t fail(sla_handle_t h, sla_status_t code, const char *fmt, const char *detail = "") {
+    if (h) snprintf(h->err, sizeof h->err, fmt, detail);
+    return code;
+}
+
+sla_status_t cuda_fail(sla_handle_t h, cudaError_t e, const char *where) {
+    if (h) snprintf(h->err, sizeof h->err, "%s: %s", where, cudaGetErrorString(e));
+    return SLA_ERR_CUDA;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks that do not depend on the call: layout and parameters.  Returns NULL when fine, else why.
+const char *check_layout_params(const sla_layout_t *l, const sla_params_t *p, bool decode) {
+    if (!l || !p) return "layout or params is NULL";
+    if (l->batch <= 0 || l->n_q_heads <= 0 || l->n_kv_heads <= 0) return "batch and head counts must be positive";
+    if (l->n_q_heads % l->n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
+    if (l->n_q_heads / l->n_kv_heads > sla::kMaxGroup) return "group size above 16";
+    if (l->head_dim != 64 && l->head_dim != 128) return "head_dim must be 64 or 128";
+    if (l->dtype != SLA_F32 && l->dtype != SLA_BF16) return "dtype must be SLA_F32 or SLA_BF16";
+    if (l->reserved != 0) return "reserved must be 0";
+    const int64_t strides[6] = {l->q_stride_b, l->q_stride_h, l->q_stride_t,
+                                l->kv_stride_b, l->kv_stride_h, l->kv_stride_t};
+    for (int j = 0; j < 6; ++j) {
+        if (decode && j == 2) continue;
+        if (strides[j] < 0 || strides[j] % 8) return "strides must be non-negative multiples of 8 elements";
+    }
+    if ((!decode && l->q_stride_t < l->head_dim) || l->kv_stride_t < l->head_dim) return "token stride below head_dim";
+    if (p->top_k < 1 || p->top_k > sla::kMaxTopK) return "top_k must be in 1..64";
+    if (p->span_len < 0 || p->back_factor < 0 || p->fwd_factor < 0) return "span_len and factors must be >= 0";
+    if (p->window < 0) return "window must be >= 0";
+    if (!(p->softmax_scale == p->softmax_scale) || !(p->search_scale == p->search_scale)) return "scale is NaN";
+    return nullptr;
+}
+
+sla_status_t check_supported(sla_handle_t h, const sla_params_t *p) {
+    if (p->window != 0) return fail(h, SLA_ERR_UNSUPPORTED, "window > 0 is not implemented%s");
+    if (p->mode != SLA_UNION) return fail(h, SLA_ERR_UNSUPPORTED, "only SLA_UNION is implemented%s");
+    return SLA_OK;
+}
+
+sla::Call make_call(const sla_handle_t h, const sla_layout_t *l, const sla_params_t *p, int64_t Lq,
+                    int64_t q_pos0, int64_t Lkv) {
+    sla::Call c;
+    c.B = l->batch; c.Hq = l->n_q_heads; c.Hkv = l->n_kv_heads; c.D = l->head_dim;
+    c.G = l->n_q_heads / l->n_kv_heads;
+    c.q_sb = l->q_stride_b; c.q_sh = l->q_stride_h; c.q_st = l->q_stride_t;
+    c.kv_sb = l->kv_stride_b; c.kv_sh = l->kv_stride_h; c.kv_st = l->kv_stride_t;
+    c.Lq = Lq; c.q_pos0 = q_pos0; c.Lkv = Lkv;
+    c.top_k = p->top_k; c.span_len = p->span_len; c.back = p->back_factor; c.fwd = p->fwd_factor;
+    c.search_scale = p->search_scale; c.softmax_scale = p->softmax_scale;
+    c.status = h ? reinterpret_cast<int *>(h->ws) : nullptr;
+    return c;
+}
+
+const char *check_prefill_range(int64_t Lq, int64_t q_pos0, int64_t Lkv) {
+    if (Lq <= 0 || q_pos0 < 0 || Lkv <= 0) return "Lq, Lkv must be positive and q_pos0 >= 0";
+    if (q_pos0 + Lq > Lkv) return "q_pos0 + Lq exceeds Lkv";
+    if (Lkv > 2147483647LL) return "Lkv above 2^31-1";
+    return nullptr;
+}
+
+size_t elem_size(int dtype) { return dtype == SLA_F32 ? 4 : 2; }
+
+}  // namespace
+
+extern "C" {
+
+const char *sla_status_string(sla_status_t s) {
+    switch (s) {
+        case SLA_OK: return "SLA_OK";
+        case SLA_ERR_INVALID_ARG: return "SLA_ERR_INVALID_ARG";
+        case SLA_ERR_UNSUPPORTED: return "SLA_ERR_UNSUPPORTED";
+        case SLA_ERR_WORKSPACE: return "SLA_ERR_WORKSPACE";
+        case SLA_ERR_CUDA: return "SLA_ERR_CUDA";
+        case SLA_ERR_DEVICE_TIMEOUT: return "SLA_ERR_DEVICE_TIMEOUT";
+        case SLA_ERR_DEVICE_INDEX: return "SLA_ERR_DEVICE_INDEX";
+    }
+    return "SLA_ERR_UNKNOWN";
+}
+
+const char *sla_last_error(sla_handle_t h) { return h ? h->err : "NULL handle"; }
+
+sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes) {
+    if (!handle) return SLA_ERR_INVALID_ARG;
+    *handle = nullptr;
+    int n_dev = 0;
+    cudaError_t e = cudaGetDeviceCount(&n_dev);
+    if (e != cudaSuccess) return SLA_ERR_CUDA;
+    if (device < 0 || device >= n_dev) return SLA_ERR_INVALID_ARG;
+    sla_handle_s *h = new (std::nothrow) sla_handle_s();
+    if (!h) return SLA_ERR_CUDA;
+    h->device = device;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device);
+    h->ws_bytes = workspace_bytes + kHeaderBytes;
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&h->ws), h->ws_bytes);
+    if (e == cudaSuccess) e = cudaMemset(h->ws, 0, kHeaderBytes);
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) {
+        if (h->ws) cudaFree(h->ws);
+        delete h;
+        return SLA_ERR_CUDA;
+    }
+    *handle = h;
+    return SLA_OK;
+}
+
+sla_status_t sla_destroy(sla_handle_t h) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    cudaError_t e = cudaFree(h->ws);
+    delete h;
+    return e == cudaSuccess ? SLA_OK : SLA_ERR_CUDA;
+}
+
+size_t sla_workspace_bytes(const sla_layout_t *l, const sla_params_t *p, int64_t Lq, int64_t Lkv) {
+    if (check_layout_params(l, p, true) || Lq <= 0 || Lkv <= 0 || Lq > Lkv) return 0;
+    sla::Call c = make_call(nullptr, l, p, Lq, Lkv - Lq, Lkv);
+    // the SM count only changes how the decode work is split; size for a generous upper bound
+    const sla::DecodePlan dp = sla::plan_decode(c, Lkv, 256 * l->batch * l->n_q_heads);
+    size_t need = dp.bytes;
+    return need + 4096;
+}
+
+sla_status_t sla_poll_status(sla_handle_t h, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, h->ws, sizeof word, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->ws, 0, sizeof word, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_poll_status");
+    if (word & sla::kStatusTimeout) return fail(h, SLA_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired%s");
+    if (word & sla::kStatusBadIndex) return fail(h, SLA_ERR_DEVICE_INDEX, "an anchor outside [0, i] was skipped%s");
+    return SLA_OK;
+}
+
+sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int64_t Lq, int64_t q_pos0,
+                             int64_t Lkv, const sla_layout_t *l, const sla_params_t *p,
+                             int32_t *out_anchor, float *out_score, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (const char *why = check_layout_params(l, p, false)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (const char *why = check_prefill_range(Lq, q_pos0, Lkv)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (!q_s || !k || !out_anchor || !out_score) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
+    if (!aligned16(q_s) || !aligned16(k)) return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
+    if (sla_status_t s = check_supported(h, p)) return s;
+    sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
+    cudaError_t e = sla::launch_search_simt(q_s, k, c, l->dtype, out_anchor, out_score,
+                                            static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_search");
+    return SLA_OK;
+}
+
+sla_status_t sla_span_attention(sla_handle_t h, const void *q, const void *k, const void *v, int64_t Lq,
+                                int64_t q_pos0, int64_t Lkv, const sla_layout_t *l, const sla_params_t *p,
+                                const int32_t *anchor, void *out, float *lse, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (const char *why = check_layout_params(l, p, false)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (const char *why = check_prefill_range(Lq, q_pos0, Lkv)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (!q || !k || !v || !anchor || !out || !lse) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
+    if (sla_status_t s = check_supported(h, p)) return s;
+    sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
+    cudaError_t e = sla::launch_attn_simt(q, k, v, c, l->dtype, anchor, out, lse,
+                                          static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_attention");
+    return SLA_OK;
+}
+
+sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, const void *k_cache,
+                             const void *v_cache, int64_t n_ctx, const sla_layout_t *l,
+                             const sla_params_t *p, void *out, float *lse, int32_t *out_anchor,
+                             float *out_score, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (const char *why = check_layout_params(l, p, true)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (n_ctx <= 0 || n_ctx > 2147483647LL) return fail(h, SLA_ERR_INVALID_ARG, "n_ctx must be in 1..2^31-1%s");
+    if (!q_s || !q || !k_cache || !v_cache || !out || !lse || !out_anchor || !out_score)
+        return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
+    if (!aligned16(q_s) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
+        return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
+    if (sla_status_t s = check_supported(h, p)) return s;
+    sla::Call c = make_call(h, l, p, 1, n_ctx - 1, n_ctx);
+    const sla::DecodePlan plan =
+        sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim));
+    if (plan.bytes + kHeaderBytes > h->ws_bytes) return fail(h, SLA_ERR_WORKSPACE, "workspace too small for this decode step%s");
+    if ((size_t)plan.n_anchor * sizeof(float) > 200 * 1024) return fail(h, SLA_ERR_UNSUPPORTED, "context too long for the decode top-k kernel%s");
+    cudaError_t e = sla::launch_decode(q_s, q, k_cache, v_cache, c, l->dtype, n_ctx, plan, h->ws + kHeaderBytes,
+                                       out, lse, out_anchor, out_score, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_decode_step");
+    return SLA_OK;
+}
+
+size_t sla_host_staging_bytes(const sla_layout_t *l, const sla_params_t *p, int64_t L) {
+    if (check_layout_params(l, p, true) || L <= 0) return 0;
+    const size_t es = elem_size(l->dtype);
+    const size_t qn = (size_t)l->batch * l->n_q_heads * L * l->head_dim;
+    const size_t kn = (size_t)l->batch * l->n_kv_heads * L * l->head_dim;
+    const size_t rows = (size_t)l->batch * l->n_q_heads * L;
+    // q_s, q, out + k, v + lse + anchors + scores, each rounded up to 256 bytes
+    return 3 * (qn * es + 256) + 2 * (kn * es + 256) + (rows * 4 + 256) + 2 * (rows * p->top_k * 4 + 256);
+}
+
+sla_status_t sla_prefill_host(sla_handle_t h, const void *q_s_host, const void *q_host, const void *k_host,
+                              const void *v_host, int64_t L, const sla_layout_t *l, const sla_params_t *p,
+                              void *out_host, float *lse_host, int32_t *anchor_host, float *score_host,
+                              void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (const char *why = check_layout_params(l, p, true)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (L <= 0 || L > 2147483647LL) return fail(h, SLA_ERR_INVALID_ARG, "L out of range%s");
+    if (!q_s_host || !q_host || !k_host || !v_host || !out_host || !lse_host || !anchor_host || !score_host)
+        return fail(h, SLA_ERR_INVALID_ARG, "NULL host pointer%s");
+    sla_layout_t dl = *l;
+    dl.q_stride_t = dl.kv_stride_t = l->head_dim;
+    dl.q_stride_h = dl.kv_stride_h = L * l->head_dim;
+    dl.q_stride_b = dl.q_stride_h * l->n_q_heads;
+    dl.kv_stride_b = dl.kv_stride_h * l->n_kv_heads;
+    const size_t work = sla_workspace_bytes(&dl, p, L, L);
+    const size_t stage = sla_host_staging_bytes(&dl, p, L);
+    if (kHeaderBytes + work + stage > h->ws_bytes) return fail(h, SLA_ERR_WORKSPACE, "workspace too small for host staging%s");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t es = elem_size(l->dtype);
+    const size_t qb = (size_t)l->batch * l->n_q_heads * L * l->head_dim * es;
+    const size_t kb = (size_t)l->batch * l->n_kv_heads * L * l->head_dim * es;
+    const size_t rows = (size_t)l->batch * l->n_q_heads * L;
+    // staging sits at the END of the workspace so that the scratch of the two steps keeps its place
+    char *base = h->ws + h->ws_bytes - stage;
+    auto take = [&base](size_t n) { char *p0 = base; base += (n + 255) & ~(size_t)255; return p0; };
+    char *d_qs = take(qb), *d_q = take(qb), *d_out = take(qb), *d_k = take(kb), *d_v = take(kb);
+    float *d_lse = (float *)take(rows * 4);
+    int32_t *d_anchor = (int32_t *)take(rows * p->top_k * 4);
+    float *d_score = (float *)take(rows * p->top_k * 4);
+    cudaError_t e = cudaMemcpyAsync(d_qs, q_s_host, qb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_k, k_host, kb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_q, q_host, qb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_v, v_host, kb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_prefill_host (copy in)");
+    sla_status_t s = sla_span_search(h, d_qs, d_k, L, 0, L, &dl, p, d_anchor, d_score, stream);
+    if (s != SLA_OK) return s;
+    s = sla_span_attention(h, d_q, d_k, d_v, L, 0, L, &dl, p, d_anchor, d_out, d_lse, stream);
+    if (s != SLA_OK) return s;
+    e = cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(lse_host, d_lse, rows * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(anchor_host, d_anchor, rows * p->top_k * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(score_host, d_score, rows * p->top_k * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_prefill_host (copy out)");
+    return SLA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,421 @@
+// Decode step of libsla (Section "Kernel design", paragraph "Decoding path"): routing scores over
+// the anchors of the single query position i = n_ctx-1, top-k, then attention over the routed spans
+// read from the KV cache.  The step is bound by HBM reads of the selected K/V rows, so the attention
+// kernel spreads each head's tokens evenly over many CTAs (split-K), streams whole rows with 16-byte
+// loads, keeps a running (max, denominator, numerator) per lane group and merges at the end.
+//
+//   decode_score   grid (anchor chunks, B*Hkv, head tiles)   K anchor rows x G routing queries
+//   decode_topk    grid (B*Hq)                               k best anchors, spans, overlap clipping
+//   decode_attn    grid (n_splits, B*Hq)                     online softmax over an even token share
+//   decode_merge   grid (B*Hq)                               log-sum-exp merge of the split results
+#include <limits.h>
+#include <math_constants.h>
+
+#include "sla_kernels.h"
+
+namespace sla {
+
+namespace {
+
+constexpr int kScoreThreads = 256;
+constexpr int kTopkThreads = 128;
+constexpr int kAttnThreads = 256;
+
+template <int LPR> __device__ inline float reduce_sub(float x) {
+#pragma unroll
+    for (int off = LPR / 2; off >= 1; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    return x;
+}
+
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D, int GT>
+__global__ void __launch_bounds__(kScoreThreads)
+decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long long n_ctx, int n,
+             float *__restrict__ scores) {
+    constexpr int E = Vec16<T>::kElems;
+    constexpr int LPR = D / E;
+    constexpr int RPI = 32 / LPR;
+    constexpr int U = 2;
+    constexpr int kWarps = kScoreThreads / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane % LPR, rsel = lane / LPR;
+    const int g = blockIdx.y % c.Hkv, b = blockIdx.y / c.Hkv;
+    const int h0 = g * c.G + blockIdx.z * GT;
+    const long long i = n_ctx - 1;
+    const T *kbase = k + b * c.kv_sb + g * c.kv_sh;
+
+    float qv[GT][E];
+#pragma unroll
+    for (int t = 0; t < GT; ++t) Vec16<T>::load(q_s + b * c.q_sb + (long long)(h0 + t) * c.q_sh + sub * E, qv[t]);
+
+    const int s_base = blockIdx.x * (kWarps * RPI * U);
+    float part[U][GT];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int s = s_base + (u * kWarps + warp) * RPI + rsel;
+#pragma unroll
+        for (int t = 0; t < GT; ++t) part[u][t] = 0.f;
+        if (s < n) {
+            const long long tpos = i + 1 - (long long)(s + 1) * (s + 1);
+            float kv[E];
+            Vec16<T>::load(kbase + tpos * c.kv_st + sub * E, kv);
+#pragma unroll
+            for (int t = 0; t < GT; ++t)
+#pragma unroll
+                for (int e = 0; e < E; ++e) part[u][t] = fmaf(qv[t][e], kv[e], part[u][t]);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int s = s_base + (u * kWarps + warp) * RPI + rsel;
+#pragma unroll
+        for (int t = 0; t < GT; ++t) {
+            const float tot = reduce_sub<LPR>(part[u][t]);
+            if (sub == 0 && s < n)
+                scores[((long long)b * c.Hq + h0 + t) * n + s] = tot * c.search_scale;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Top-k of one head's anchor scores (largest first, smaller stride index on ties), the spans of the
+// selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)]) sorted and clipped to disjoint
+// pieces, and their cumulative token counts.
+__global__ void __launch_bounds__(kTopkThreads)
+decode_topk(Call c, long long n_ctx, int n, const float *__restrict__ scores, int *__restrict__ spans,
+            int32_t *__restrict__ out_anchor, float *__restrict__ out_score) {
+    extern __shared__ float sc[];
+    __shared__ float wv[kTopkThreads / 32];
+    __shared__ int ws[kTopkThreads / 32];
+    __shared__ int s_lo[kMaxTopK], s_hi[kMaxTopK], p_lo[kMaxTopK], p_hi[kMaxTopK];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const long long bh = blockIdx.x;
+    const long long i = n_ctx - 1;
+    const float *src = scores + bh * n;
+    for (int s = tid; s < n; s += kTopkThreads) sc[s] = src[s];
+    __syncthreads();
+
+    for (int j = 0; j < c.top_k; ++j) {
+        float bv = -CUDART_INF_F;
+        int bs = INT_MAX;
+        for (int s = tid; s < n; s += kTopkThreads) {
+            const float v = sc[s];
+            if (v > bv) { bv = v; bs = s; }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+            const int os = __shfl_xor_sync(0xffffffffu, bs, off);
+            if (ov > bv || (ov == bv && os < bs)) { bv = ov; bs = os; }
+        }
+        if (lane == 0) { wv[warp] = bv; ws[warp] = bs; }
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 1; w < kTopkThreads / 32; ++w)
+                if (wv[w] > bv || (wv[w] == bv && ws[w] < bs)) { bv = wv[w]; bs = ws[w]; }
+            int lo = INT_MAX, hi = -1;
+            if (bs != INT_MAX) {
+                const long long t = i + 1 - (long long)(bs + 1) * (bs + 1);
+                out_anchor[bh * c.top_k + j] = (int32_t)t;
+                out_score[bh * c.top_k + j] = bv;
+                sc[bs] = -CUDART_INF_F;
+                const long long ell = base_len(i, c.span_len);
+                const long long a = t - (long long)c.back * ell, z = t + (long long)c.fwd * ell;
+                lo = (int)(a > 0 ? a : 0);
+                hi = (int)(z < i ? z : i);
+            } else {
+                out_anchor[bh * c.top_k + j] = -1;
+                out_score[bh * c.top_k + j] = -CUDART_INF_F;
+            }
+            s_lo[j] = lo;
+            s_hi[j] = hi;
+        }
+        __syncthreads();
+    }
+    // rank sort by (lo, hi, index), then clip overlaps into disjoint pieces
+    if (tid < c.top_k) {
+        const int lo = s_lo[tid], hi = s_hi[tid];
+        int rank = 0;
+        for (int m = 0; m < c.top_k; ++m) {
+            const int lm = s_lo[m], hm = s_hi[m];
+            rank += (lm < lo) || (lm == lo && (hm < hi || (hm == hi && m < tid)));
+        }
+        p_lo[rank] = lo;
+        p_hi[rank] = hi;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int *start = spans + bh * (2 * c.top_k + 2);
+        int *cum = start + c.top_k;
+        int cnt = 0;
+        long long next_free = 0, total = 0;
+        cum[0] = 0;
+        for (int a = 0; a < c.top_k; ++a) {
+            const int lo = p_lo[a], hi = p_hi[a];
+            if (hi < 0) break;
+            const long long j0 = lo > next_free ? lo : next_free;
+            if (j0 <= hi) {
+                start[cnt] = (int)j0;
+                total += hi - j0 + 1;
+                cum[cnt + 1] = (int)total;
+                ++cnt;
+            }
+            if ((long long)hi + 1 > next_free) next_free = (long long)hi + 1;
+        }
+        start[2 * c.top_k + 1] = cnt;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(kAttnThreads)
+decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, Call c,
+            const int *__restrict__ spans, float *__restrict__ partial) {
+    constexpr int E = Vec16<T>::kElems;
+    constexpr int LPR = D / E;
+    constexpr int RPI = 32 / LPR;
+    constexpr int U = 4;
+    constexpr int kWarps = kAttnThreads / 32;
+    constexpr int kSlots = kWarps * RPI;  // token rows the CTA reads per load step
+    __shared__ int s_start[kMaxTopK], s_cum[kMaxTopK + 1];
+    __shared__ float s_m[kSlots], s_l[kSlots];
+    __shared__ float s_acc[kWarps][D];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane % LPR, rsel = lane / LPR;
+    const long long bh = blockIdx.y;
+    const int h = (int)(bh % c.Hq), b = (int)(bh / c.Hq), g = h / c.G;
+    const int n_splits = gridDim.x, split = blockIdx.x;
+
+    const int *sp = spans + bh * (2 * c.top_k + 2);
+    const int cnt = sp[2 * c.top_k + 1];
+    for (int j = tid; j < cnt; j += kAttnThreads) s_start[j] = sp[j];
+    for (int j = tid; j <= cnt; j += kAttnThreads) s_cum[j] = sp[c.top_k + j];
+    __syncthreads();
+    const long long total = cnt > 0 ? s_cum[cnt] : 0;
+    const long long f_begin = total * split / n_splits, f_end = total * (split + 1) / n_splits;
+
+    const T *kbase = k + b * c.kv_sb + g * c.kv_sh;
+    const T *vbase = v + b * c.kv_sb + g * c.kv_sh;
+    float qv[E];
+    Vec16<T>::load(q + b * c.q_sb + (long long)h * c.q_sh + sub * E, qv);
+    const float scale2 = c.softmax_scale * kLog2e;
+#pragma unroll
+    for (int e = 0; e < E; ++e) qv[e] *= scale2;
+
+    float m = -CUDART_INF_F, l = 0.f, acc[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    int piece = 0;
+    const int slot = warp * RPI + rsel;
+
+    for (long long f0 = f_begin; f0 < f_end; f0 += kSlots * U) {
+        uint4 kraw[U], vraw[U];
+        bool ok[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long f = f0 + u * kSlots + slot;
+            ok[u] = f < f_end;
+            if (ok[u]) {
+                while (f >= s_cum[piece + 1]) ++piece;
+                const long long pos = s_start[piece] + (f - s_cum[piece]);
+                kraw[u] = __ldg(reinterpret_cast<const uint4 *>(kbase + pos * c.kv_st + sub * E));
+                vraw[u] = __ldg(reinterpret_cast<const uint4 *>(vbase + pos * c.kv_st + sub * E));
+            } else {
+                kraw[u] = make_uint4(0, 0, 0, 0);
+                vraw[u] = make_uint4(0, 0, 0, 0);
+            }
+        }
+        float x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            float kv[E];
+            if constexpr (sizeof(T) == 2) {
+                Vec16<__nv_bfloat16>::unpack(kraw[u], kv);
+            } else {
+                kv[0] = __uint_as_float(kraw[u].x); kv[1] = __uint_as_float(kraw[u].y);
+                kv[2] = __uint_as_float(kraw[u].z); kv[3] = __uint_as_float(kraw[u].w);
+            }
+            x[u] = 0.f;
+#pragma unroll
+            for (int e = 0; e < E; ++e) x[u] = fmaf(qv[e], kv[e], x[u]);
+        }
+        float m_new = m;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            x[u] = reduce_sub<LPR>(x[u]);
+            if (ok[u]) m_new = fmaxf(m_new, x[u]);
+        }
+        const float r = (m == -CUDART_INF_F) ? 0.f : exp2f(m - m_new);
+        l *= r;
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] *= r;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const float p = ok[u] ? exp2f(x[u] - m_new) : 0.f;
+            l += p;
+            float vv[E];
+            if constexpr (sizeof(T) == 2) {
+                Vec16<__nv_bfloat16>::unpack(vraw[u], vv);
+            } else {
+                vv[0] = __uint_as_float(vraw[u].x); vv[1] = __uint_as_float(vraw[u].y);
+                vv[2] = __uint_as_float(vraw[u].z); vv[3] = __uint_as_float(vraw[u].w);
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[e] = fmaf(p, vv[e], acc[e]);
+        }
+        m = m_new;
+    }
+
+    // merge the lane groups of the warp, then the warps of the CTA
+#pragma unroll
+    for (int off = LPR; off < 32; off <<= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, off);
+        const float ol = __shfl_xor_sync(0xffffffffu, l, off);
+        const float mn = fmaxf(m, om);
+        const float a = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
+        const float bb = (om == -CUDART_INF_F) ? 0.f : exp2f(om - mn);
+        l = l * a + ol * bb;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const float oa = __shfl_xor_sync(0xffffffffu, acc[e], off);
+            acc[e] = acc[e] * a + oa * bb;
+        }
+        m = mn;
+    }
+    if (rsel == 0) {
+        if (sub == 0) { s_m[warp] = m; s_l[warp] = l; }
+#pragma unroll
+        for (int e = 0; e < E; ++e) s_acc[warp][sub * E + e] = acc[e];
+    }
+    __syncthreads();
+    if (tid < D) {
+        float mm = -CUDART_INF_F;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) mm = fmaxf(mm, s_m[w]);
+        float ll = 0.f, aa = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float sc = (s_m[w] == -CUDART_INF_F) ? 0.f : exp2f(s_m[w] - mm);
+            ll += s_l[w] * sc;
+            aa += s_acc[w][tid] * sc;
+        }
+        float *dst = partial + (bh * n_splits + split) * (D + 2);
+        if (tid == 0) { dst[0] = mm; dst[1] = ll; }
+        dst[2 + tid] = aa;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(D)
+decode_merge(Call c, int n_splits, const float *__restrict__ partial, T *__restrict__ out,
+             float *__restrict__ lse) {
+    const long long bh = blockIdx.x;
+    const int h = (int)(bh % c.Hq), b = (int)(bh / c.Hq), d = threadIdx.x;
+    const float *src = partial + bh * n_splits * (D + 2);
+    float mm = -CUDART_INF_F;
+    for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, src[s * (D + 2)]);
+    float ll = 0.f, aa = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        const float ms = src[s * (D + 2)];
+        const float sc = (ms == -CUDART_INF_F) ? 0.f : exp2f(ms - mm);
+        ll += src[s * (D + 2) + 1] * sc;
+        aa += src[s * (D + 2) + 2 + d] * sc;
+    }
+    out[b * c.q_sb + (long long)h * c.q_sh + d] = from_float<T>(ll > 0.f ? aa / ll : 0.f);
+    if (d == 0) lse[bh] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
+}
+
+template <typename T, int D>
+cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const void *v, const Call &c,
+                          long long n_ctx, const DecodePlan &p, void *scratch, void *out, float *lse,
+                          int32_t *out_anchor, float *out_score, cudaStream_t st) {
+    constexpr int E = Vec16<T>::kElems;
+    constexpr int RPI = 32 / (D / E);
+    char *base = (char *)scratch;
+    float *scores = (float *)(base + p.off_scores);
+    int *spans = (int *)(base + p.off_spans);
+    float *partial = (float *)(base + p.off_partial);
+    const int n = p.n_anchor;
+    const int rows_per_cta = (kScoreThreads / 32) * RPI * 2;
+    const int gt = c.G % 8 == 0 ? 8 : c.G % 4 == 0 ? 4 : c.G % 2 == 0 ? 2 : 1;
+    dim3 gs((n + rows_per_cta - 1) / rows_per_cta, c.B * c.Hkv, c.G / gt);
+    const T *qs = (const T *)q_s, *kk = (const T *)k;
+    switch (gt) {
+        case 8: decode_score<T, D, 8><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, scores); break;
+        case 4: decode_score<T, D, 4><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, scores); break;
+        case 2: decode_score<T, D, 2><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, scores); break;
+        default: decode_score<T, D, 1><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, scores); break;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t smem = (size_t)n * sizeof(float);
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    if (smem > 48 * 1024) {
+        e = cudaFuncSetAttribute(decode_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    decode_topk<<<c.B * c.Hq, kTopkThreads, smem, st>>>(c, n_ctx, n, scores, spans, out_anchor, out_score);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    decode_attn<T, D><<<dim3(p.n_splits, c.B * c.Hq), kAttnThreads, 0, st>>>(
+        (const T *)q, kk, (const T *)v, c, spans, partial);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    decode_merge<T, D><<<c.B * c.Hq, D, 0, st>>>(c, p.n_splits, partial, (T *)out, lse);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int decode_attn_blocks_per_sm(int dtype, int D) {
+    static int cache[2][2] = {{0, 0}, {0, 0}};
+    int &slot = cache[dtype == SLA_F32 ? 0 : 1][D == 64 ? 0 : 1];
+    if (slot == 0) {
+        int n = 0;
+        cudaError_t e;
+        if (dtype == SLA_F32)
+            e = D == 64 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<float, 64>, kAttnThreads, 0)
+                        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<float, 128>, kAttnThreads, 0);
+        else
+            e = D == 64 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<__nv_bfloat16, 64>, kAttnThreads, 0)
+                        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<__nv_bfloat16, 128>, kAttnThreads, 0);
+        slot = (e == cudaSuccess && n > 0) ? n : 1;
+    }
+    return slot;
+}
+
+DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots) {
+    DecodePlan p;
+    p.n_anchor = (int)isqrt_ll(n_ctx);
+    const long long ell = base_len(n_ctx - 1, c.span_len);
+    long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
+    if (span_tokens > n_ctx) span_tokens = n_ctx;
+    const long long max_tokens = span_tokens * c.top_k;
+    // one resident wave: as many splits per head as fit the CTA slots of the device
+    long long ns = (long long)cta_slots / ((long long)c.B * c.Hq);
+    if (ns > max_tokens / 128) ns = max_tokens / 128;
+    if (ns > 256) ns = 256;
+    if (ns < 1) ns = 1;
+    p.n_splits = (int)ns;
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t bh = (size_t)c.B * c.Hq;
+    p.off_scores = 0;
+    p.off_spans = align(p.off_scores + bh * (size_t)p.n_anchor * sizeof(float));
+    p.off_partial = align(p.off_spans + bh * (size_t)(2 * c.top_k + 2) * sizeof(int));
+    p.bytes = align(p.off_partial + bh * (size_t)p.n_splits * (c.D + 2) * sizeof(float));
+    return p;
+}
+
+cudaError_t launch_decode(const void *q_s, const void *q, const void *k, const void *v, const Call &c,
+                          int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, void *out,
+                          float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st) {
+    if (dtype == SLA_F32) {
+        return c.D == 64 ? decode_launch<float, 64>(q_s, q, k, v, c, n_ctx, plan, scratch, out, lse, out_anchor, out_score, st)
+                         : decode_launch<float, 128>(q_s, q, k, v, c, n_ctx, plan, scratch, out, lse, out_anchor, out_score, st);
+    }
+    return c.D == 64 ? decode_launch<__nv_bfloat16, 64>(q_s, q, k, v, c, n_ctx, plan, scratch, out, lse, out_anchor, out_score, st)
+                     : decode_launch<__nv_bfloat16, 128>(q_s, q, k, v, c, n_ctx, plan, scratch, out, lse, out_anchor, out_score, st);
+}
+
+}  // namespace sla

@@ -1,0 +1,31 @@
+// Internal launcher declarations of libsla (the public interface is include/sla.h).
+#pragma once
+
+#include "sla_common.cuh"
+
+namespace sla {
+
+// ---- generic SIMT kernels (sla_simt.cu) --------------------------------------------------------
+cudaError_t launch_search_simt(const void *q_s, const void *k, const Call &c, int dtype,
+                               int32_t *out_anchor, float *out_score, cudaStream_t st);
+cudaError_t launch_attn_simt(const void *q, const void *k, const void *v, const Call &c, int dtype,
+                             const int32_t *anchor, void *out, float *lse, cudaStream_t st);
+
+// ---- decode step (sla_decode.cu) ---------------------------------------------------------------
+// Scratch layout of one decode step, all offsets in bytes from the scratch base.
+struct DecodePlan {
+    int n_anchor;       // anchors of the query position, floor(sqrt(n_ctx))
+    int n_splits;       // CTAs that share one query head's tokens
+    size_t off_scores;  // float [B*Hq][n_anchor]
+    size_t off_spans;   // int   [B*Hq][2*top_k + 2]: piece start, cumulative token offset, total, count
+    size_t off_partial; // float [B*Hq][n_splits][D + 2]: running max, denominator, numerator
+    size_t bytes;
+};
+// cta_slots = SM count x resident decode_attn CTAs per SM (see decode_attn_blocks_per_sm)
+DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots);
+int decode_attn_blocks_per_sm(int dtype, int D);
+cudaError_t launch_decode(const void *q_s, const void *q, const void *k, const void *v, const Call &c,
+                          int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, void *out,
+                          float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st);
+
+}  // namespace sla

@@ -1,0 +1,179 @@
+"""GPU parity, small cases: the CUDA path (through the C-ABI binding) against the fp64 oracle,
+element by element, on sizes that span several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import parity_util as P
+from oracle import sla_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sla():
+    import paper_2601_18401_b200 as sla_pkg
+    return sla_pkg
+
+
+@pytest.fixture(scope="module")
+def handle(sla):
+    h = sla.Handle(0, 1 << 30)
+    yield h
+    h.close()
+
+
+def workload(**kw):
+    from paper_2601_18401_b200 import synth
+    base = synth.Workload("t", "prefill", 1, 4, 2, 128, 1000, "bf16", 16, 4, seed=77)
+    return base.scaled(**kw)
+
+
+def run_prefill(sla, handle, w, q_pos0=0, Lq=None, permute=False, softmax_scale=None, search_scale=1.0):
+    from paper_2601_18401_b200 import synth
+    x = synth.make_prefill(w, device="cuda:0")
+    if permute:  # [B,L,H,D] storage viewed as [B,H,L,D]: non-trivial strides
+        x = {n: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) for n, t in x.items()}
+    L = w.seq_len
+    Lq = L - q_pos0 if Lq is None else Lq
+    params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim,
+                             softmax_scale=softmax_scale, search_scale=search_scale)
+    q_s = x["q_s"][:, :, q_pos0:q_pos0 + Lq]
+    q = x["q"][:, :, q_pos0:q_pos0 + Lq]
+    anchor, score = sla.sla_span_search(handle, q_s, x["k"], params, q_pos0=q_pos0)
+    out, lse = sla.sla_span_attention(handle, q, x["k"], x["v"], anchor, params, q_pos0=q_pos0)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    host = P.host_inputs({"q_s": q_s, "q": q, "k": x["k"], "v": x["v"]})
+    code = synth.dtype_code(w.dtype)
+    ref_s = O.span_search(host["q_s"], host["k"], code, top_k=w.top_k, q_pos0=q_pos0, search_scale=search_scale)
+    ties = P.compare_search(anchor, score, ref_s, q_pos0=q_pos0)
+    ref_a = P.oracle_attention_for(host, code, anchor, w, q_pos0=q_pos0, softmax_scale=softmax_scale)
+    err, lerr = P.compare_attention(out, lse, ref_a, w.dtype)
+    return dict(ties=ties, err=err, lerr=lerr, anchor=anchor, out=out, lse=lse, host=host, ref_a=ref_a)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(),                                                                  # bf16 D128 GQA, ragged L
+    dict(dtype="f32"),                                                       # fp32 D128
+    dict(head_dim=64, n_q_heads=2, n_kv_heads=2),                            # bf16 D64 MHA
+    dict(dtype="f32", head_dim=64, n_q_heads=3, n_kv_heads=1, seq_len=777),  # odd group size
+    dict(span_len=0, back_factor=4, fwd_factor=2, top_k=2),                  # paper rule l(i), extended factors
+    dict(batch=2, n_q_heads=8, n_kv_heads=1, seq_len=1537, span_len=33, top_k=7),
+    dict(top_k=40, seq_len=300, span_len=5),                                 # more slots than anchors: padding
+    dict(top_k=1, span_len=100, seq_len=2100),
+    dict(back_factor=0, fwd_factor=0, span_len=7),                           # single-token spans
+    dict(seq_len=1, top_k=3), dict(seq_len=2, top_k=3), dict(seq_len=5, top_k=2),
+])
+def test_prefill_parity(sla, handle, kw):
+    run_prefill(sla, handle, workload(**kw))
+
+
+def test_prefill_chunk_and_strides(sla, handle):
+    w = workload(seq_len=1800, span_len=21, top_k=5)
+    run_prefill(sla, handle, w, q_pos0=1111)                  # last chunk
+    run_prefill(sla, handle, w, q_pos0=640, Lq=500)           # middle chunk
+    run_prefill(sla, handle, w, permute=True)                 # [B,L,H,D] storage
+    run_prefill(sla, handle, w, softmax_scale=0.05, search_scale=0.5)
+
+
+def test_tiny_config_full_and_dense(sla, handle):
+    """First benchmark configuration in full (fp32, L=4096, l=64): k=4 against the oracle, and
+    k=64 (every anchor) against dense causal attention computed here with numpy."""
+    from paper_2601_18401_b200 import synth
+    w = synth.CONFIGS[0]
+    res = run_prefill(sla, handle, w)
+    assert res["err"] <= 1e-4
+    r = run_prefill(sla, handle, w.scaled(top_k=64))
+    q, k, v = (r["host"][n][0, 0].astype(np.float64) for n in ("q", "k", "v"))
+    x = (q @ k.T) / np.sqrt(w.head_dim)
+    x = np.where(np.tril(np.ones_like(x, dtype=bool)), x, -np.inf)
+    m = x.max(axis=1, keepdims=True)
+    e = np.exp(x - m)
+    dense = (e / e.sum(axis=1, keepdims=True)) @ v
+    got = r["out"].float().cpu().numpy()[0, 0]
+    assert np.abs(got - dense).max() <= 1e-4
+    lse = (m[:, 0] + np.log(e.sum(axis=1)))
+    assert np.abs(r["lse"].cpu().numpy()[0, 0] - lse).max() <= 1e-4
+
+
+def test_attention_with_foreign_anchors(sla, handle):
+    """Anchors need not come from span-search: duplicates, -1 holes, arbitrary positions <= i."""
+    from paper_2601_18401_b200 import synth
+    w = workload(seq_len=900, span_len=25, top_k=6)
+    x = synth.make_prefill(w, device="cuda:0")
+    g = torch.Generator().manual_seed(3)
+    i = torch.arange(w.seq_len)
+    anchor = (torch.rand(1, 4, w.seq_len, 6, generator=g) * (i[None, None, :, None] + 1)).long().clamp(max=w.seq_len - 1)
+    anchor = torch.minimum(anchor, i[None, None, :, None].expand_as(anchor))
+    anchor[..., 1] = anchor[..., 0]            # duplicate
+    anchor[..., 2] = -1                        # hole
+    anchor[:, :, 100:120] = -1                 # rows without any anchor
+    anchor = anchor.to(torch.int32).cuda()
+    params = sla.make_params(6, 25, head_dim=128)
+    out, lse = sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    ref = P.oracle_attention_for(P.host_inputs(x), O.BF16, anchor, w)
+    P.compare_attention(out, lse, ref, "bf16")
+    assert torch.all(out[:, :, 100:120] == 0) and torch.all(torch.isinf(lse[:, :, 100:120]))
+    # an anchor beyond the query position is skipped and reported, never dereferenced
+    anchor[0, 0, 10, 0] = 500
+    out2, _ = sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == -6
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+
+
+@pytest.mark.parametrize("dtype,D,Hq,Hkv", [("bf16", 128, 8, 2), ("f32", 64, 2, 2), ("bf16", 64, 4, 1), ("f32", 128, 3, 1)])
+def test_decode_parity(sla, handle, dtype, D, Hq, Hkv):
+    from paper_2601_18401_b200 import synth
+    cap = 70100
+    w = synth.Workload("d", "decode", 2, Hq, Hkv, D, 70000, dtype, 60, 6, steps=4, seed=5)
+    kc, vc = synth.make_decode_cache(w, "cuda:0", capacity=cap)
+    hk, hv = synth.to_numpy(kc), synth.to_numpy(vc)
+    code = synth.dtype_code(dtype)
+    for n_ctx, span_len, top_k in [(1, 60, 6), (2, 60, 6), (3, 0, 2), (10, 2, 3), (1000, 0, 4), (4097, 64, 8),
+                                   (70000, 60, 6), (70000, 0, 16), (65536, 300, 64)]:
+        step = synth.make_decode_step_inputs(w, n_ctx, "cuda:0")
+        params = sla.make_params(top_k, span_len, head_dim=D)
+        out, lse, anchor, score = sla.sla_decode_step(handle, step["q_s"], step["q"], kc, vc, n_ctx, params)
+        torch.cuda.synchronize()
+        ref = O.decode_step(synth.to_numpy(step["q_s"]), synth.to_numpy(step["q"]), hk, hv, code,
+                            n_ctx=n_ctx, top_k=top_k, span_len=span_len)
+        rs = {k_: ref[k_][:, :, None] for k_ in ("anchor", "score", "gap")}
+        P.compare_search(anchor[:, :, None], score[:, :, None], rs, q_pos0=n_ctx - 1)
+        ref2 = O.decode_step(synth.to_numpy(step["q_s"]), synth.to_numpy(step["q"]), hk, hv, code,
+                             n_ctx=n_ctx, top_k=top_k, span_len=span_len)
+        # attention parity on the GPU's own anchors
+        att = O.span_attention(synth.to_numpy(step["q"])[:, :, None], hk, hv, code,
+                               anchor.cpu().numpy()[:, :, None], span_len=span_len, q_pos0=n_ctx - 1, Lkv=n_ctx)
+        P.compare_attention(out[:, :, None], lse[:, :, None], att, dtype)
+        del ref2
+
+
+def test_error_returns(sla, handle):
+    from paper_2601_18401_b200 import synth
+    w = workload(seq_len=64)
+    x = synth.make_prefill(w, device="cuda:0")
+    with pytest.raises(sla.SlaError) as e:
+        sla.sla_span_search(handle, x["q_s"], x["k"], sla.make_params(4, 16, window=8))
+    assert e.value.status == -2
+    with pytest.raises(sla.SlaError) as e:
+        sla.sla_span_search(handle, x["q_s"], x["k"], sla.make_params(0, 16))
+    assert e.value.status == -1
+    with pytest.raises(sla.SlaError) as e:
+        sla.sla_span_search(handle, x["q_s"], x["k"], sla.make_params(4, 16), q_pos0=10)
+    assert e.value.status == -1
+    with pytest.raises(sla.SlaError) as e:
+        sla.sla_span_attention(handle, x["q"], x["k"], x["v"],
+                               torch.zeros(1, 4, 64, 4, dtype=torch.int32, device="cuda"),
+                               sla.make_params(4, 16, mode=sla.SLA_PER_SPAN))
+    assert e.value.status == -2
+    small = sla.Handle(0, 1024)
+    kc = torch.zeros(1, 2, 100000, 128, dtype=torch.bfloat16, device="cuda")
+    qq = torch.zeros(1, 4, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(sla.SlaError) as e:
+        sla.sla_decode_step(small, qq, qq, kc, kc, 100000, sla.make_params(4, 16))
+    assert e.value.status == -3
+    small.close()
