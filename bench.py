@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the span-search + span-attention hot path on B200.
+
+One "step" is one pass of the prefill hot path -- sla_span_search followed by sla_span_attention --
+over one batch of seeded synthetic input of the second benchmark configuration (batch 1, 32 query /
+8 KV heads, head_dim 128, L = 65536, bf16, 16 planted key spans per head, span length 256, top_k 8).
+The headline value is prefill tokens/s per attention layer with the inputs resident in HBM; the
+same run also measures the end-to-end figure through the host-buffer C call, the decode step at
+1M and 10M context (microseconds per token per layer), the roofline fractions, and the CPU oracle
+on a bounded sample as a baseline.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched under torchrun, one rank per GPU) every rank runs the same workload on its own
+sequence -- the path shards over independent sequences with no exchange step -- and the value is
+the total over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2601_18401_b200 import synth
+
+METRIC = "prefill_tokens_per_s_per_layer"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+# ------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons in the background during the timed region."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        busy = sorted(sm)[len(sm) // 2:] if sm else []   # upper half: samples taken under load
+        return {"sm_mhz": float(np.median(busy)) if busy else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------ bookkeeping
+def attended_pairs(anchor: torch.Tensor, span_len: int, back: int, fwd: int) -> int:
+    """(query, key) pairs the union of the selected spans holds -- bookkeeping for the FLOP count
+    (4 * head_dim per pair), computed with torch ops from the anchors the search produced."""
+    B, H, L, K = anchor.shape
+    i = torch.arange(L, device=anchor.device, dtype=torch.int64)[None, None, :, None]
+    t = anchor.to(torch.int64)
+    lo = torch.clamp(t - back * span_len, min=0)
+    hi = torch.minimum(t + fwd * span_len, i.expand_as(t))
+    valid = t >= 0
+    lo = torch.where(valid, lo, torch.full_like(lo, 1 << 40))
+    hi = torch.where(valid, hi, torch.full_like(hi, -1))
+    lo, order = torch.sort(lo, dim=-1)
+    hi = torch.gather(hi, -1, order)
+    run_hi = torch.cummax(hi, dim=-1).values
+    prev = torch.cat([torch.full_like(run_hi[..., :1], -1), run_hi[..., :-1]], dim=-1)
+    start = torch.maximum(lo, prev + 1)
+    return int(torch.clamp(hi - start + 1, min=0).sum().item())
+
+
+def oracle_sample_rows(L: int, n: int):
+    return np.unique(np.linspace(0, L - 1, n).astype(np.int64))
+
+
+def time_oracle_prefill(w, host, rows):
+    """Runs the CPU oracle (search + attention) on `rows` of every head; returns seconds."""
+    from oracle import sla_oracle as O
+    code = synth.dtype_code(w.dtype)
+    t0 = time.perf_counter()
+    s = O.span_search(host["q_s"], host["k"], code, top_k=w.top_k, rows=rows)
+    O.span_attention(host["q"], host["k"], host["v"], code, s["anchor"], span_len=w.span_len,
+                     back_factor=w.back_factor, fwd_factor=w.fwd_factor, rows=rows)
+    return time.perf_counter() - t0
+
+
+# ------------------------------------------------------------------------------------ arms
+def run_reference(args, w):
+    """The CPU oracle as it stands, on host cores, on a bounded row sample per step."""
+    from oracle import sla_oracle as O
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    x = synth.make_prefill(w, device="cpu")
+    host = {n: synth.to_numpy(t) for n, t in x.items()}
+    rows = oracle_sample_rows(w.seq_len, args.ref_rows)
+    for _ in range(args.warmup):
+        time_oracle_prefill(w, host, rows[: max(4, len(rows) // 16)])
+    secs = [time_oracle_prefill(w, host, rows) for _ in range(args.steps)]
+    per_step = float(np.mean(secs))
+    value = len(rows) * w.batch / per_step
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
+                   "head_dim": w.head_dim, "seq_len": w.seq_len, "span_len": w.span_len, "top_k": w.top_k},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
+                         "sample": f"{len(rows)} evenly spaced query positions x all {w.n_q_heads} heads per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def bench_decode(sla, handle, w, steps, peaks, dev):
+    """Decode loop: append the new token's K/V, then one sla_decode_step, `steps` times."""
+    kc, vc = synth.make_decode_cache(w, dev, capacity=w.seq_len + steps + 8)
+    params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim)
+    ins = [synth.make_decode_step_inputs(w, s, dev) for s in range(8)]
+    out = sla.sla_decode_step(handle, ins[0]["q_s"], ins[0]["q"], kc, vc, w.seq_len, params)
+
+    def one(step):
+        x = ins[step % len(ins)]
+        n_ctx = w.seq_len + step + 1
+        kc[:, :, n_ctx - 1] = x["k_new"]
+        vc[:, :, n_ctx - 1] = x["v_new"]
+        sla.sla_decode_step(handle, x["q_s"], x["q"], kc, vc, n_ctx, params, out=out[0], lse=out[1],
+                            out_anchor=out[2], out_score=out[3])
+    for s in range(5):
+        one(s)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for s in range(steps):
+        one(s)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / steps
+    # kernel-only: the decode call alone, same cache, back to back
+    e0.record()
+    for s in range(steps):
+        x = ins[s % len(ins)]
+        sla.sla_decode_step(handle, x["q_s"], x["q"], kc, vc, w.seq_len + steps, params, out=out[0], lse=out[1],
+                            out_anchor=out[2], out_score=out[3])
+    e1.record()
+    torch.cuda.synchronize()
+    us_call = e0.elapsed_time(e1) * 1e3 / steps
+    # tokens of the de-duplicated union of the selected spans (bookkeeping for the byte count)
+    anchor = out[2].to(torch.int64)
+    i = w.seq_len + steps - 1
+    lo = torch.clamp(anchor - w.back_factor * w.span_len, min=0)
+    hi = torch.clamp(anchor + w.fwd_factor * w.span_len, max=i)
+    lo, order = torch.sort(lo, dim=-1)
+    hi = torch.gather(hi, -1, order)
+    run_hi = torch.cummax(hi, dim=-1).values
+    prev = torch.cat([torch.full_like(run_hi[..., :1], -1), run_hi[..., :-1]], dim=-1)
+    pairs = int(torch.clamp(hi - torch.maximum(lo, prev + 1) + 1, min=0).sum().item())
+    elem = 2 if w.dtype == "bf16" else 4
+    n_anchor = int(np.floor(np.sqrt(w.seq_len + steps)))
+    bytes_step = pairs * 2 * w.head_dim * elem + n_anchor * w.batch * w.n_kv_heads * w.head_dim * elem
+    gbs = bytes_step / (us_call * 1e-6) / 1e9
+    del kc, vc
+    torch.cuda.empty_cache()
+    return {"workload": w.name, "us_per_token_per_layer": us, "us_per_decode_call": us_call, "steps": steps,
+            "algorithmic_bytes_per_step": bytes_step,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0,
+                         "traffic": None, "peak_source": peaks["_source"]}}
+
+
+def run_ours(args, w):
+    import paper_2601_18401_b200 as sla
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    sla.load_library()
+    peaks = load_peaks()
+
+    wr = w.scaled(seed=w.seed + 7919 * rank)      # every rank its own sequence
+    x = synth.make_prefill(wr, device=dev)
+    params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim)
+    layout = sla.make_layout(x["q"], x["k"])
+    work = sla.sla_workspace_bytes(layout, params, w.seq_len, w.seq_len)
+    stage = sla.sla_host_staging_bytes(layout, params, w.seq_len)
+    handle = sla.Handle(local, work + stage + (64 << 20))
+    B, Hq, L, D = x["q"].shape
+    anchor = torch.empty(B, Hq, L, w.top_k, dtype=torch.int32, device=dev)
+    score = torch.empty(B, Hq, L, w.top_k, dtype=torch.float32, device=dev)
+    out = torch.empty_like(x["q"])
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
+
+    def step(ev=None):
+        sla.sla_span_search(handle, x["q_s"], x["k"], params, out_anchor=anchor, out_score=score)
+        if ev is not None:
+            ev[0].record()
+        sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params, out=out, lse=lse)
+        if ev is not None:
+            ev[1].record()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    launches0 = sla.sla_kernel_launches(handle)
+    sampler = ClockSampler(local)
+    sampler.start()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for s in range(args.steps):
+        step(evs[s])
+    t1.record()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    clocks = sampler.stop()
+    launches = sla.sla_kernel_launches(handle) - launches0
+    total_ms = t0.elapsed_time(t1)
+    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    if dist:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * B * L / (ms_per_step * 1e-3)
+
+    # roofline of the dominant kernel (span-attention): 4*D flops per attended (query, key) pair
+    pairs = attended_pairs(anchor, w.span_len, w.back_factor, w.fwd_factor)
+    flops = 4.0 * D * pairs
+    tflops = flops / (attn_ms * 1e-3) / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"]
+    roofline = {"bound": "tensor", "kernel": "sla_span_attention", "achieved": tflops, "peak": peak_tf,
+                "unit": "TFLOP/s", "frac": tflops / peak_tf, "traffic": None, "flops_per_launch": flops,
+                "ms_per_launch": attn_ms, "search_ms_per_launch": ms_per_step - attn_ms,
+                "peak_source": peaks["_source"] + " (sustained bf16 matmul)"}
+
+    # end to end through the host-buffer C call: pinned host inputs, host outputs, copies inside
+    host = {n: t.cpu().pin_memory() for n, t in x.items()}
+    ho = sla.sla_prefill_host(handle, host["q_s"], host["q"], host["k"], host["v"], params)
+    n_e2e = max(2, min(args.steps, 5))
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    tt = time.perf_counter()
+    for _ in range(n_e2e):
+        sla.sla_prefill_host(handle, host["q_s"], host["q"], host["k"], host["v"], params,
+                             out=ho[0], lse=ho[1], anchor=ho[2], score=ho[3])
+    e2e_s = (time.perf_counter() - tt) / n_e2e
+    if dist:
+        t = torch.tensor([e2e_s], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    h2d = sum(host[n].numel() * host[n].element_size() for n in ("q_s", "q", "k", "v"))
+    d2h = sum(t.numel() * t.element_size() for t in ho)
+    e2e = {"value": world * B * L / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "ms_per_step": e2e_s * 1e3}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "batch_per_gpu": B, "q_heads": Hq, "kv_heads": w.n_kv_heads, "head_dim": D,
+                   "seq_len": L, "span_len": w.span_len, "top_k": w.top_k, "back_factor": w.back_factor,
+                   "fwd_factor": w.fwd_factor, "planted_spans": w.planted_spans,
+                   "l2": "inputs (1.3 GB) exceed the 126 MB L2; no flush between steps",
+                   "parallelism": f"independent sequences x{world}"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+    }
+
+    if rank == 0 and not args.no_decode:
+        del x, anchor, score, out, lse
+        torch.cuda.empty_cache()
+        dec = []
+        for ci, steps in ((3, 256), (4, 128)):
+            try:
+                dec.append(bench_decode(sla, handle, synth.CONFIGS[ci], steps if not args.quick else 16, peaks, dev))
+            except torch.cuda.OutOfMemoryError as e:  # pragma: no cover
+                dec.append({"workload": synth.CONFIGS[ci].name, "skipped": f"out of memory: {e}"})
+        line["decode"] = dec
+    if rank == 0 and not args.no_cpu_baseline:
+        from oracle import sla_oracle as O
+        rows = oracle_sample_rows(L, args.ref_rows)
+        hn = {n: synth.to_numpy(t) for n, t in host.items()}
+        secs = time_oracle_prefill(w, hn, rows)
+        line["cpu_baseline"] = {"value": len(rows) * B / secs, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
+                                "sample": f"{len(rows)} evenly spaced query positions x all {Hq} heads, "
+                                          f"search + attention, {secs:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=1, help="index into the benchmark configurations (prefill ones)")
+    ap.add_argument("--ref-rows", type=int, default=1024, help="query positions the CPU oracle is timed on")
+    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true", help="short decode loops (for smoke runs)")
+    args = ap.parse_args()
+    w = synth.CONFIGS[args.workload]
+    if w.kind != "prefill":
+        raise SystemExit("--workload must name a prefill configuration; decode is reported alongside")
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

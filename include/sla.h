@@ -119,6 +119,10 @@ const char *sla_last_error(sla_handle_t handle);    /* text of the last failure 
  * SLA_ERR_DEVICE_INDEX; the word is cleared. */
 sla_status_t sla_poll_status(sla_handle_t handle, void *stream);
 
+/* Number of kernels this handle has launched since sla_create (a diagnostic for benchmarks; the
+ * paper has no counterpart).  Host-only. */
+int64_t sla_kernel_launches(sla_handle_t handle);
+
 /* ---- span-search (Section "Span search"; Algorithm 1 scoring and TopK lines) -------------- */
 
 /* Query row r (0 <= r < Lq) is position i = q_pos0 + r; keys 0 .. Lkv-1 are valid; requires

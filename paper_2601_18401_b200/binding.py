@@ -23,7 +23,7 @@ SLA_UNION, SLA_PER_SPAN = 0, 1
 EXPORTS = [
     "sla_create", "sla_destroy", "sla_workspace_bytes", "sla_status_string", "sla_last_error",
     "sla_poll_status", "sla_span_search", "sla_span_attention", "sla_decode_step",
-    "sla_host_staging_bytes", "sla_prefill_host",
+    "sla_host_staging_bytes", "sla_prefill_host", "sla_kernel_launches",
 ]
 
 
@@ -79,6 +79,8 @@ def load_library():
     lib.sla_span_attention.argtypes = [vp, vp, vp, vp, i64, i64, i64, LP, PP, vp, vp, vp, vp]
     lib.sla_decode_step.restype = i32
     lib.sla_decode_step.argtypes = [vp, vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
+    lib.sla_kernel_launches.restype = i64
+    lib.sla_kernel_launches.argtypes = [vp]
     lib.sla_host_staging_bytes.restype = sz
     lib.sla_host_staging_bytes.argtypes = [LP, PP, i64]
     lib.sla_prefill_host.restype = i32
@@ -160,6 +162,10 @@ def sla_workspace_bytes(layout: sla_layout_t, params: sla_params_t, Lq: int, Lkv
 
 def sla_host_staging_bytes(layout: sla_layout_t, params: sla_params_t, L: int) -> int:
     return int(load_library().sla_host_staging_bytes(C.byref(layout), C.byref(params), int(L)))
+
+
+def sla_kernel_launches(handle: Handle) -> int:
+    return int(handle._lib.sla_kernel_launches(handle.ptr))
 
 
 def sla_poll_status(handle: Handle, stream=None) -> int:

@@ -12,6 +12,7 @@ struct sla_handle_s {
     int sm_count = 0;
     char *ws = nullptr;       // device workspace; the first kHeaderBytes hold the status word
     size_t ws_bytes = 0;
+    long long launches = 0;   // kernels launched through this handle
     char err[256] = {0};
 };
 
@@ -102,6 +103,8 @@ const char *sla_status_string(sla_status_t s) {
 
 const char *sla_last_error(sla_handle_t h) { return h ? h->err : "NULL handle"; }
 
+int64_t sla_kernel_launches(sla_handle_t h) { return h ? h->launches : 0; }
+
 sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes) {
     if (!handle) return SLA_ERR_INVALID_ARG;
     *handle = nullptr;
@@ -171,6 +174,7 @@ sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int
     cudaError_t e = sla::launch_search_simt(q_s, k, c, l->dtype, out_anchor, out_score,
                                             static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_search");
+    h->launches += 1;
     return SLA_OK;
 }
 
@@ -188,6 +192,7 @@ sla_status_t sla_span_attention(sla_handle_t h, const void *q, const void *k, co
     cudaError_t e = sla::launch_attn_simt(q, k, v, c, l->dtype, anchor, out, lse,
                                           static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_attention");
+    h->launches += 1;
     return SLA_OK;
 }
 
@@ -211,6 +216,7 @@ sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, con
     cudaError_t e = sla::launch_decode(q_s, q, k_cache, v_cache, c, l->dtype, n_ctx, plan, h->ws + kHeaderBytes,
                                        out, lse, out_anchor, out_score, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_decode_step");
+    h->launches += 4;
     return SLA_OK;
 }
 
