@@ -1,6 +1,7 @@
 // Host side of libsla: handle, argument validation, workspace carving and kernel dispatch.
 // Every exported function is declared and documented in include/sla.h.
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -13,6 +14,8 @@ struct sla_handle_s {
     char *ws = nullptr;       // device workspace; the first kHeaderBytes hold the status word
     size_t ws_bytes = 0;
     long long launches = 0;   // kernels launched through this handle
+    size_t scratch_avail = 0; // bytes of workspace after the header that kernels may use as scratch
+    bool force_simt = false;  // environment SLA_FORCE_SIMT=1: generic kernels only (for A/B checks)
     char err[256] = {0};
 };
 
@@ -120,6 +123,8 @@ sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes
     e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device);
     h->ws_bytes = workspace_bytes + kHeaderBytes;
+    h->scratch_avail = workspace_bytes;
+    if (const char *fs = getenv("SLA_FORCE_SIMT")) h->force_simt = fs[0] == '1';
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&h->ws), h->ws_bytes);
     if (e == cudaSuccess) e = cudaMemset(h->ws, 0, kHeaderBytes);
     cudaSetDevice(prev);
@@ -145,6 +150,11 @@ size_t sla_workspace_bytes(const sla_layout_t *l, const sla_params_t *p, int64_t
     // the SM count only changes how the decode work is split; size for a generous upper bound
     const sla::DecodePlan dp = sla::plan_decode(c, Lkv, 256 * l->batch * l->n_q_heads);
     size_t need = dp.bytes;
+    if (sla::tc_attention_shape_ok(c, l->dtype)) {
+        // tensor-core span-attention: scratch for chunks of up to 65536 query positions
+        const sla::TcPlan tp = sla::plan_attention_tc(c, (int)(Lq < 65536 ? Lq : 65536));
+        if (tp.bytes > need) need = tp.bytes;
+    }
     return need + 4096;
 }
 
@@ -189,8 +199,18 @@ sla_status_t sla_span_attention(sla_handle_t h, const void *q, const void *k, co
         return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
     if (sla_status_t s = check_supported(h, p)) return s;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
-    cudaError_t e = sla::launch_attn_simt(q, k, v, c, l->dtype, anchor, out, lse,
-                                          static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!h->force_simt && sla::tc_attention_supported(c, l->dtype)) {
+        // tensor-core path; needs scratch for at least a modest chunk of query positions
+        const long long min_chunk = Lq < 1024 ? Lq : 1024;
+        if (sla::plan_attention_tc(c, (int)min_chunk).bytes <= h->scratch_avail) {
+            cudaError_t e = sla::launch_attn_tc(q, k, v, c, anchor, out, lse, h->ws + kHeaderBytes,
+                                                h->scratch_avail, h->sm_count, st, &h->launches);
+            if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_attention (tensor-core path)");
+            return SLA_OK;
+        }
+    }
+    cudaError_t e = sla::launch_attn_simt(q, k, v, c, l->dtype, anchor, out, lse, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_attention");
     h->launches += 1;
     return SLA_OK;
@@ -264,9 +284,11 @@ sla_status_t sla_prefill_host(sla_handle_t h, const void *q_s_host, const void *
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_q, q_host, qb, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_v, v_host, kb, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_prefill_host (copy in)");
+    const size_t avail_before = h->scratch_avail;
+    h->scratch_avail = h->ws_bytes - kHeaderBytes - stage;   // the staging buffers are not scratch
     sla_status_t s = sla_span_search(h, d_qs, d_k, L, 0, L, &dl, p, d_anchor, d_score, stream);
-    if (s != SLA_OK) return s;
-    s = sla_span_attention(h, d_q, d_k, d_v, L, 0, L, &dl, p, d_anchor, d_out, d_lse, stream);
+    if (s == SLA_OK) s = sla_span_attention(h, d_q, d_k, d_v, L, 0, L, &dl, p, d_anchor, d_out, d_lse, stream);
+    h->scratch_avail = avail_before;
     if (s != SLA_OK) return s;
     e = cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(lse_host, d_lse, rows * 4, cudaMemcpyDeviceToHost, st);

@@ -1,0 +1,750 @@
+// Tensor-core span-attention for prefill (bf16, head_dim 128): tcgen05 MMA with TMEM accumulators,
+// K/V tiles by TMA, one softmax thread per query row.
+//
+// What it computes is Section "Span attention" (A_{i,t} = Attention(Q(i), K[S_t], V[S_t])) with the
+// spans of Algorithm 1, under union semantics: the k spans of a (query, head) row are sorted and
+// clipped to disjoint "pieces"; every piece is attended on its own and the per-piece results are
+// merged exactly through their log-sum-exp.
+//
+// The systems problem (Section "Kernel design"): neighbouring queries pick different spans, so the
+// rows of one MMA tile must be made to share a key footprint.  Here pieces are grouped by the
+// 64-key block their right end falls in (per batch and KV head) and, inside a group, ordered by how
+// many key blocks they cover, with one counting sort (histogram, prefix sum, scatter) -- no
+// comparison sort of the queries.  A tile is 128 pieces of one group: their Q rows are gathered into
+// shared memory and the tile walks the key blocks they cover from left to right.
+//
+//   tc_pieces<count>     per row: spans -> pieces, histogram of (group, blocks covered)
+//   tc_scan              prefix sums, tile table
+//   tc_pieces<scatter>   per row: piece records to their sorted places
+//   tc_attend            persistent CTAs, tiles handed out through an atomic counter; per tile and
+//                        key block: S = Q K^T (tcgen05, smem x smem -> TMEM), row softmax in
+//                        registers, P (bf16) back into TMEM, O += P V (tcgen05, TMEM x smem -> TMEM)
+//   tc_merge             per row: log-sum-exp merge of its pieces -> out, lse
+//
+// CTA layout of tc_attend (192 threads, two CTAs per SM): warps 0-3 own one tile row each (TMEM lane
+// = row): Q gather, softmax, epilogue; warp 4 issues the MMAs; warp 5 issues the TMA loads.  TMEM:
+// two 64-column S buffers (P aliases the S it came from) and 128 columns of O.  Every wait on an
+// mbarrier is bounded; when one runs out the CTA raises a status bit, drains and leaves.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <cuda_fp16.h>
+#include <limits.h>
+#include <math_constants.h>
+
+#include "sla_kernels.h"
+#include "sla_tc_ptx.cuh"
+
+namespace sla {
+
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int kD = 128;
+constexpr int kBK = 64;          // keys per block
+constexpr int kRows = 128;       // pieces per tile
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 256;
+constexpr uint32_t kColS = 0;    // S buffers at columns 0 and 64
+constexpr uint32_t kColO = 128;
+constexpr int kQBytes = kRows * kD * 2;      // 32 KiB, two 64-wide halves of 128 rows x 128 B
+constexpr int kKVBytes = kBK * kD * 2;       // 16 KiB, two 64-wide halves of 64 rows x 128 B
+constexpr int kOffQ = 0;
+constexpr int kOffK = kQBytes;
+constexpr int kOffV = kOffK + 2 * kKVBytes;
+constexpr int kOffMeta = kOffV + 2 * kKVBytes;   // 98304
+constexpr int kMetaBytes = 2048;
+constexpr int kSmemBytes = kOffMeta + kMetaBytes + 1024;  // + slack for 1024-byte alignment
+constexpr float kRescaleThreshold = 8.f;     // log2 units: P stays below 2^8
+
+struct Meta {
+    unsigned long long q_full, o_full;
+    unsigned long long kv_full[2], kv_empty[2], s_full[2], p_ready[2];
+    uint32_t tmem_base;
+    int tile;
+    int sb_min;
+    int abort_flag;
+    int lo[kRows];
+    int hi[kRows];
+};
+static_assert(sizeof(Meta) <= kMetaBytes, "meta block too large");
+
+struct TcParams {
+    const bf16 *q;
+    long long q_sb, q_sh, q_st;
+    int Hq, G, Lc, top_k;
+    long long r0;              // first query row of the chunk
+    float scale2;              // softmax_scale * log2(e)
+    int slot_t, slot_h, slot_b;  // positions of (token, head, batch) among tensor-map coordinates 1..3
+    const int4 *recs;          // sorted piece records {row, j, lo, hi}
+    const int4 *tiles;         // {b*Hkv+g, end block, first record, record count}
+    const int *n_tiles;
+    int *tile_counter;
+    __half *part_o;            // [rows*top_k][128] normalised piece outputs, fp16 with one power-of-two
+                               // scale per 32-column chunk (block floating point)
+    float2 *part_lse;          // [rows*top_k] {log2-domain log-sum-exp of the piece, four chunk exponents}
+    int *status;
+    int Hkv;
+};
+
+// ------------------------------------------------------------------------------------------------
+// Pieces of one row: spans of the selected anchors (Algorithm 1), sorted by (lo, hi), clipped so
+// that each key is kept once.  Returns the number of pieces; lo[]/hi[] hold them left to right.
+__device__ inline int row_pieces(const int32_t *__restrict__ an, int top_k, long long i, long long ell,
+                                 int back, int fwd, int *lo, int *hi, int *status) {
+    int n = 0;
+    for (int j = 0; j < top_k; ++j) {
+        const long long t = an[j];
+        if (t > i) { atomicOr(status, kStatusBadIndex); continue; }
+        if (t < 0) continue;
+        const long long a = t - (long long)back * ell, z = t + (long long)fwd * ell;
+        const int l0 = (int)(a > 0 ? a : 0), h0 = (int)(z < i ? z : i);
+        int pos = n;   // insertion sort by (lo, hi)
+        while (pos > 0 && (lo[pos - 1] > l0 || (lo[pos - 1] == l0 && hi[pos - 1] > h0))) {
+            lo[pos] = lo[pos - 1];
+            hi[pos] = hi[pos - 1];
+            --pos;
+        }
+        lo[pos] = l0;
+        hi[pos] = h0;
+        ++n;
+    }
+    int cnt = 0;
+    long long next_free = 0;
+    for (int a = 0; a < n; ++a) {
+        const int l0 = lo[a], h0 = hi[a];
+        const long long j0 = l0 > next_free ? l0 : next_free;
+        if (j0 <= h0) {
+            lo[cnt] = (int)j0;
+            hi[cnt] = h0;
+            ++cnt;
+        }
+        if ((long long)h0 + 1 > next_free) next_free = (long long)h0 + 1;
+    }
+    return cnt;
+}
+
+struct PrepParams {
+    const int32_t *anchor;  // [B,Hq,Lq,top_k]
+    int B, Hq, Hkv, G, top_k, span_len, back, fwd;
+    long long Lq, q_pos0, r0;
+    int Lc;                 // query rows of this chunk (per head)
+    int NB, nb_max;         // key blocks, largest number of blocks a piece may cover
+    int *key_count;         // [n_keys] histogram, later the exclusive offsets
+    int *key_cursor;        // [n_keys]
+    int4 *recs;
+    unsigned char *n_pieces;  // [rows]
+    int *status;
+};
+
+// One thread per (b, h, r) row of the chunk.  kScatter = false: count; true: write the records.
+template <bool kScatter>
+__global__ void __launch_bounds__(128) tc_pieces(PrepParams p) {
+    const long long row = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long rows = (long long)p.B * p.Hq * p.Lc;
+    if (row >= rows) return;
+    const int rc = (int)(row % p.Lc);
+    const int bh = (int)(row / p.Lc);
+    const int h = bh % p.Hq, b = bh / p.Hq, g = h / p.G;
+    const long long r = p.r0 + rc;
+    const long long i = p.q_pos0 + r;
+    int lo[kMaxTopK], hi[kMaxTopK];
+    const int32_t *an = p.anchor + (((long long)b * p.Hq + h) * p.Lq + r) * p.top_k;
+    const int cnt = row_pieces(an, p.top_k, i, base_len(i, p.span_len), p.back, p.fwd, lo, hi, p.status);
+    if (!kScatter) p.n_pieces[row] = (unsigned char)cnt;
+    const long long group0 = ((long long)b * p.Hkv + g) * p.NB;
+    for (int j = 0; j < cnt; ++j) {
+        const int eb = hi[j] / kBK, sb = lo[j] / kBK;
+        const long long key = (group0 + eb) * p.nb_max + (eb - sb);
+        if (!kScatter) {
+            atomicAdd(p.key_count + key, 1);
+        } else {
+            const int pos = p.key_count[key] + atomicAdd(p.key_cursor + key, 1);
+            p.recs[pos] = make_int4((int)row, j, lo[j], hi[j]);
+        }
+    }
+}
+
+// Single block: exclusive prefix sum of the key histogram (in place), tiles per group, tile table.
+__global__ void __launch_bounds__(1024)
+tc_scan(int *key_count, long long n_keys, int nb_max, int n_groups, int NB, int4 *tiles, int *n_tiles,
+        int *tile_counter, int max_tiles) {
+    __shared__ int warp_sum[32];
+    __shared__ int carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    auto block_excl_scan = [&](int v, int &total) -> int {
+        int x = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, x, off);
+            if (lane >= off) x += y;
+        }
+        if (lane == 31) warp_sum[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            int w = warp_sum[lane];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, w, off);
+                if (lane >= off) w += y;
+            }
+            warp_sum[lane] = w;
+        }
+        __syncthreads();
+        total = warp_sum[31];
+        const int base = warp > 0 ? warp_sum[warp - 1] : 0;
+        __syncthreads();
+        return base + x - v;
+    };
+    // pass 1: key offsets
+    const long long per = (n_keys + 1023) / 1024;
+    const long long k0 = per * tid, k1 = (k0 + per < n_keys) ? k0 + per : n_keys;
+    int local = 0;
+    for (long long k = k0; k < k1; ++k) local += key_count[k];
+    int total;
+    int run = block_excl_scan(local, total);
+    for (long long k = k0; k < k1; ++k) {
+        const int c = key_count[k];
+        key_count[k] = run;
+        run += c;
+    }
+    __syncthreads();
+    const int n_recs = total;
+    // pass 2: tiles per group (a group's records are contiguous: keys group*nb_max .. +nb_max-1)
+    if (tid == 0) carry_s = 0;
+    __syncthreads();
+    for (int g0 = 0; g0 < n_groups; g0 += 1024) {
+        const int g = g0 + tid;
+        int first = 0, cnt = 0;
+        if (g < n_groups) {
+            first = key_count[(long long)g * nb_max];
+            const int last = (g + 1 < n_groups) ? key_count[(long long)(g + 1) * nb_max] : n_recs;
+            cnt = last - first;
+        }
+        const int nt = (cnt + kRows - 1) / kRows;
+        int tot;
+        const int off = block_excl_scan(nt, tot) + carry_s;
+        for (int t = 0; t < nt; ++t) {
+            const int idx = off + t;
+            if (idx < max_tiles) {
+                const int left = cnt - t * kRows;
+                tiles[idx] = make_int4(g / NB, g % NB, first + t * kRows, left < kRows ? left : kRows);
+            }
+        }
+        __syncthreads();
+        if (tid == 0) carry_s += tot;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        *n_tiles = carry_s < max_tiles ? carry_s : max_tiles;
+        *tile_counter = 0;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = ptx::smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw);
+    Meta *meta = reinterpret_cast<Meta *>(smem + kOffMeta);
+    volatile int *abort_flag = &meta->abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    const uint32_t bar_q_full = ptx::smem_u32(&meta->q_full), bar_o_full = ptx::smem_u32(&meta->o_full);
+    const uint32_t bar_kv_full = ptx::smem_u32(&meta->kv_full[0]), bar_kv_empty = ptx::smem_u32(&meta->kv_empty[0]);
+    const uint32_t bar_s_full = ptx::smem_u32(&meta->s_full[0]), bar_p_ready = ptx::smem_u32(&meta->p_ready[0]);
+
+    if (tid == 0) {
+        ptx::mbar_init(bar_q_full, kRows);
+        ptx::mbar_init(bar_o_full, 1);
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(bar_kv_full + 8 * s, 1);
+            ptx::mbar_init(bar_kv_empty + 8 * s, 1);
+            ptx::mbar_init(bar_s_full + 8 * s, 1);
+            ptx::mbar_init(bar_p_ready + 8 * s, kRows);
+        }
+        meta->abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    if (warp == 5 && lane == 0) {
+        ptx::prefetch_tensormap(&tm_k);
+        ptx::prefetch_tensormap(&tm_v);
+    }
+    if (warp == 4) {
+        ptx::tmem_alloc(ptx::smem_u32(&meta->tmem_base), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = meta->tmem_base;
+
+    constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(kRows, kBK, false, false);   // S = Q K^T, both K-major
+    constexpr uint32_t kIdescO = ptx::idesc_bf16_f32(kRows, kD, false, true);     // O = P V, V is N-major
+
+    uint32_t n_kv = 0;    // key blocks processed so far by this CTA (stage / buffer = n & 1)
+    uint32_t n_tile = 0;  // tiles processed so far
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) {
+            int t = -1;
+            if (!*abort_flag) {
+                t = atomicAdd(p.tile_counter, 1);
+                if (t >= *p.n_tiles) t = -1;
+            }
+            meta->tile = t;
+            meta->sb_min = INT_MAX;
+        }
+        __syncthreads();
+        const int tile = meta->tile;
+        if (tile < 0) break;
+        const int4 ti = p.tiles[tile];   // {b*Hkv+g, end block, first record, count}
+
+        // ---- rows of the tile (warps 0-3, one row per thread)
+        int4 rec = make_int4(0, 0, INT_MAX, -1);
+        if (warp < 4) {
+            if (tid < ti.w) rec = p.recs[ti.z + tid];
+            meta->lo[tid] = rec.z;
+            meta->hi[tid] = rec.w;
+            int sb = tid < ti.w ? rec.z / kBK : INT_MAX;
+            sb = __reduce_min_sync(0xffffffffu, sb);
+            if (lane == 0) atomicMin(&meta->sb_min, sb);
+        }
+        __syncthreads();
+        const int sb0 = meta->sb_min;
+        const int nblk = ti.y - sb0 + 1;
+        const int g = ti.x % p.Hkv, b = ti.x / p.Hkv;
+
+        if (warp == 5) {
+            // ---------------- TMA producer
+            if (lane == 0) {
+                int c[4];
+                c[1 + p.slot_h] = g;
+                c[1 + p.slot_b] = b;
+                for (int j = 0; j < nblk; ++j) {
+                    const uint32_t n = n_kv + j, st = n & 1u, ph = (n >> 1) & 1u;
+                    if (!ptx::mbar_wait(bar_kv_empty + 8 * st, ph ^ 1u, abort_flag)) break;
+                    ptx::mbar_arrive_expect_tx(bar_kv_full + 8 * st, 2 * kKVBytes);
+                    c[1 + p.slot_t] = (sb0 + j) * kBK;
+                    const uint32_t dk = base + kOffK + st * kKVBytes, dv = base + kOffV + st * kKVBytes;
+                    ptx::tma_load_4d(dk, &tm_k, bar_kv_full + 8 * st, 0, c[1], c[2], c[3]);
+                    ptx::tma_load_4d(dk + kKVBytes / 2, &tm_k, bar_kv_full + 8 * st, 64, c[1], c[2], c[3]);
+                    ptx::tma_load_4d(dv, &tm_v, bar_kv_full + 8 * st, 0, c[1], c[2], c[3]);
+                    ptx::tma_load_4d(dv + kKVBytes / 2, &tm_v, bar_kv_full + 8 * st, 64, c[1], c[2], c[3]);
+                }
+            }
+        } else if (warp == 4) {
+            // ---------------- MMA issuer: S(0); S(1), PV(0); S(2), PV(1); ...
+            if (lane == 0) {
+                bool ok = ptx::mbar_wait(bar_q_full, n_tile & 1u, abort_flag);
+                ptx::tc_fence_after();
+                for (int step = 0; ok && step <= nblk; ++step) {
+                    if (step < nblk) {
+                        const uint32_t n = n_kv + step, st = n & 1u, ph = (n >> 1) & 1u;
+                        ok = ptx::mbar_wait(bar_kv_full + 8 * st, ph, abort_flag);
+                        if (!ok) break;
+                        ptx::tc_fence_after();
+                        const uint32_t d_s = tmem + kColS + st * kBK;
+#pragma unroll
+                        for (int ks = 0; ks < kD / 16; ++ks) {
+                            const uint32_t half = ks >> 2, inner = (ks & 3) * 32;
+                            const uint64_t da = ptx::smem_desc_sw128(base + kOffQ + half * (kQBytes / 2) + inner, 16, 1024);
+                            const uint64_t db = ptx::smem_desc_sw128(base + kOffK + st * kKVBytes + half * (kKVBytes / 2) + inner, 16, 1024);
+                            ptx::mma_ss(d_s, da, db, kIdescS, ks > 0);
+                        }
+                        ptx::mma_commit(bar_s_full + 8 * st);
+                    }
+                    if (step >= 1) {
+                        const int jj = step - 1;
+                        const uint32_t n = n_kv + jj, st = n & 1u, ph = (n >> 1) & 1u;
+                        ok = ptx::mbar_wait(bar_p_ready + 8 * st, ph, abort_flag);
+                        if (!ok) break;
+                        ptx::tc_fence_after();
+                        const uint32_t a_p = tmem + kColS + st * kBK;   // P aliases S: 64 bf16 = 32 columns
+#pragma unroll
+                        for (int ks = 0; ks < kBK / 16; ++ks) {
+                            const uint64_t db = ptx::smem_desc_sw128(base + kOffV + st * kKVBytes + ks * 2048, kKVBytes / 2, 1024);
+                            ptx::mma_ts(tmem + kColO, a_p + ks * 8, db, kIdescO, (jj > 0 || ks > 0) ? 1u : 0u);
+                        }
+                        ptx::mma_commit(bar_kv_empty + 8 * st);
+                        if (jj == nblk - 1) ptx::mma_commit(bar_o_full);
+                    }
+                }
+            }
+        } else {
+            // ---------------- row threads: Q gather, softmax per key block, epilogue
+            const bool valid = tid < ti.w;
+            const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+            {
+                uint4 *qdst = reinterpret_cast<uint4 *>(smem + kOffQ);
+                if (valid) {
+                    const int rc = rec.x % p.Lc, bh = rec.x / p.Lc;
+                    const int h = bh % p.Hq, bb = bh / p.Hq;
+                    const uint4 *src = reinterpret_cast<const uint4 *>(p.q + bb * p.q_sb + h * p.q_sh + (p.r0 + rc) * p.q_st);
+                    uint4 v[16];
+#pragma unroll
+                    for (int cidx = 0; cidx < 16; ++cidx) v[cidx] = __ldg(src + cidx);
+#pragma unroll
+                    for (int cidx = 0; cidx < 16; ++cidx) {
+                        const int half = cidx >> 3, ch = (cidx & 7) ^ (tid & 7);
+                        qdst[half * (kQBytes / 32) + tid * 8 + ch] = v[cidx];
+                    }
+                } else {
+#pragma unroll
+                    for (int cidx = 0; cidx < 16; ++cidx)
+                        qdst[(cidx >> 3) * (kQBytes / 32) + tid * 8 + (cidx & 7)] = make_uint4(0, 0, 0, 0);
+                }
+                ptx::fence_proxy_async_smem();
+                ptx::mbar_arrive(bar_q_full);
+            }
+            const int lo = rec.z, hi = rec.w;
+            float m_ref = -CUDART_INF_F, l = 0.f;
+            bool ok = true;
+            for (int j = 0; j < nblk && ok; ++j) {
+                const uint32_t n = n_kv + j, st = n & 1u, ph = (n >> 1) & 1u;
+                ok = ptx::mbar_wait_warp(bar_s_full + 8 * st, ph, abort_flag);
+                if (!ok) break;
+                ptx::tc_fence_after();
+                const uint32_t s_addr = lane_addr + kColS + st * kBK;
+                uint32_t sr[2][32];
+                ptx::tmem_ld32(s_addr, sr[0]);
+                ptx::tmem_ld32(s_addr + 32, sr[1]);
+                ptx::tmem_wait_ld();
+                const int k0 = (sb0 + j) * kBK;
+                const bool any = valid && k0 <= hi && k0 + kBK - 1 >= lo;
+                const bool full = any && k0 >= lo && k0 + kBK - 1 <= hi;
+                float bm = -CUDART_INF_F;
+                if (any) {
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf)
+#pragma unroll
+                        for (int cc = 0; cc < 32; ++cc) {
+                            float x = __uint_as_float(sr[hlf][cc]) * p.scale2;
+                            if (!full) {
+                                const int kp = k0 + hlf * 32 + cc;
+                                x = (kp >= lo && kp <= hi) ? x : -CUDART_INF_F;
+                            }
+                            sr[hlf][cc] = __float_as_uint(x);
+                            bm = fmaxf(bm, x);
+                        }
+                }
+                // running reference maximum; O is rescaled only when it moves by more than the threshold
+                const bool first = (l == 0.f);   // no key of this row seen so far
+                const bool need = !first && (bm > m_ref + kRescaleThreshold);
+                if (__any_sync(0xffffffffu, need)) {
+                    // PV of the previous block must have landed before O is touched
+                    const uint32_t np = n - 1u;
+                    ok = ptx::mbar_wait_warp(bar_kv_empty + 8 * (np & 1u), (np >> 1) & 1u, abort_flag);
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    const float f = need ? ex2_approx(m_ref - bm) : 1.f;
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t o[32];
+                        ptx::tmem_ld32(lane_addr + kColO + q4 * 32, o);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
+                        ptx::tmem_st32(lane_addr + kColO + q4 * 32, o);
+                    }
+                    if (need) { l *= f; m_ref = bm; }
+                }
+                if (first && bm > -CUDART_INF_F) m_ref = bm;   // first keys of this row
+                uint32_t pk[32];
+                if (any && bm > -CUDART_INF_F) {
+                    float sum = 0.f;
+#pragma unroll
+                    for (int cc = 0; cc < 32; ++cc) {
+                        const int hlf = cc >> 4, c2 = (cc & 15) * 2;
+                        const float p0 = ex2_approx(__uint_as_float(sr[hlf][c2]) - m_ref);
+                        const float p1 = ex2_approx(__uint_as_float(sr[hlf][c2 + 1]) - m_ref);
+                        sum += p0 + p1;
+                        const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+                        pk[cc] = *reinterpret_cast<const uint32_t *>(&pp);
+                    }
+                    l += sum;
+                } else {
+#pragma unroll
+                    for (int cc = 0; cc < 32; ++cc) pk[cc] = 0u;
+                }
+                ptx::tmem_st32(s_addr, pk);
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(bar_p_ready + 8 * st);
+            }
+            // epilogue: normalised piece output and its log-sum-exp
+            if (ok) ok = ptx::mbar_wait_warp(bar_o_full, n_tile & 1u, abort_flag);
+            if (ok) {
+                ptx::tc_fence_after();
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+                const long long slot = (long long)rec.x * p.top_k + rec.y;
+                uint4 *dst = reinterpret_cast<uint4 *>(p.part_o + slot * kD);
+                uint32_t exps = 0;   // biased exponent of each 32-column chunk's largest magnitude
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t o[32];
+                    ptx::tmem_ld32(lane_addr + kColO + q4 * 32, o);
+                    ptx::tmem_wait_ld();
+                    if (valid) {
+                        float amax = 0.f;
+#pragma unroll
+                        for (int cc = 0; cc < 32; ++cc) {
+                            const float x = __uint_as_float(o[cc]) * inv;
+                            o[cc] = __float_as_uint(x);
+                            amax = fmaxf(amax, fabsf(x));
+                        }
+                        uint32_t eb = (__float_as_uint(amax) >> 23) & 0xffu;
+                        eb = eb < 1u ? 1u : (eb > 252u ? 252u : eb);
+                        exps |= eb << (8 * q4);
+                        const float down = __uint_as_float((253u - eb) << 23);   // 2^(126 - eb): chunk into [-1, 1]
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __half2 pp = __floats2half2_rn(__uint_as_float(o[v4 * 8 + 2 * e]) * down,
+                                                                     __uint_as_float(o[v4 * 8 + 2 * e + 1]) * down);
+                                w[e] = *reinterpret_cast<const uint32_t *>(&pp);
+                            }
+                            dst[q4 * 4 + v4] = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                }
+                if (valid)
+                    p.part_lse[slot] = make_float2(l > 0.f ? m_ref + log2f(l) : -CUDART_INF_F, __uint_as_float(exps));
+                ptx::tc_fence_before();
+            }
+        }
+        n_kv += nblk;
+        n_tile += 1;
+    }
+
+    // ---- teardown
+    __syncthreads();
+    if (*abort_flag) {
+        if (tid == 0) atomicOr(p.status, kStatusTimeout);
+        __nanosleep(200000);   // let copies and MMAs that may still be in flight land
+        __syncthreads();
+    }
+    if (warp == 4) {
+        __syncwarp();
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Per row: merge the normalised piece outputs through their log-sum-exp.  16 threads per row.
+__global__ void __launch_bounds__(256)
+tc_merge(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
+         const unsigned char *__restrict__ n_pieces, Call c, int Lc, long long r0, bf16 *__restrict__ out,
+         float *__restrict__ lse) {
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long row = gid >> 4;
+    const int sub = (int)(gid & 15);
+    const long long rows = (long long)c.B * c.Hq * Lc;
+    if (row >= rows) return;
+    const int cnt = n_pieces[row];
+    const float2 *pl = part_lse + row * c.top_k;
+    float mx = -CUDART_INF_F;
+    for (int j = 0; j < cnt; ++j) mx = fmaxf(mx, pl[j].x);
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    float den = 0.f;
+    if (mx > -CUDART_INF_F) {
+        for (int j = 0; j < cnt; ++j) {
+            const float2 pj = pl[j];
+            if (pj.x == -CUDART_INF_F) continue;
+            const float w = exp2f(pj.x - mx);
+            den += w;
+            const uint32_t eb = (__float_as_uint(pj.y) >> (8 * (sub >> 2))) & 0xffu;
+            const float ws = w * __uint_as_float((eb + 1u) << 23);   // weight x 2^(eb - 126)
+            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(part_o + (row * c.top_k + j) * kD + sub * 8));
+            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&rw[e]));
+                acc[2 * e] = fmaf(ws, f.x, acc[2 * e]);
+                acc[2 * e + 1] = fmaf(ws, f.y, acc[2 * e + 1]);
+            }
+        }
+    }
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    const int rc = (int)(row % Lc);
+    const int bh = (int)(row / Lc);
+    const int h = bh % c.Hq, b = bh / c.Hq;
+    const long long r = r0 + rc;
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 pp = __floats2bfloat162_rn(acc[2 * e] * inv, acc[2 * e + 1] * inv);
+        w[e] = *reinterpret_cast<const uint32_t *>(&pp);
+    }
+    *reinterpret_cast<uint4 *>(out + b * c.q_sb + h * c.q_sh + r * c.q_st + sub * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+    if (sub == 0)
+        lse[((long long)b * c.Hq + h) * c.Lq + r] = den > 0.f ? (mx + log2f(den)) * kLn2 : -CUDART_INF_F;
+}
+
+// ------------------------------------------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+    }
+    return fn;
+}
+
+// Tensor map over K or V [B, Hkv, Lkv, 128] with arbitrary (16-byte aligned) strides; the three outer
+// dimensions are ordered by ascending stride, slot[] says where (token, head, batch) ended up.
+bool make_kv_map(CUtensorMap *tm, const void *ptr, const Call &c, int slot[3]) {
+    auto fn = encode_fn();
+    if (!fn) return false;
+    struct Dim { unsigned long long size, stride; int which; };
+    Dim d[3] = {{(unsigned long long)c.Lkv, (unsigned long long)c.kv_st * 2, 0},
+                {(unsigned long long)c.Hkv, (unsigned long long)c.kv_sh * 2, 1},
+                {(unsigned long long)c.B, (unsigned long long)c.kv_sb * 2, 2}};
+    for (int a = 0; a < 3; ++a)
+        for (int bq = a + 1; bq < 3; ++bq) {
+            const bool swap = (d[bq].size > 1 && d[a].size == 1) ? false
+                              : (d[a].size > 1 && d[bq].size == 1) ? false
+                              : d[bq].stride < d[a].stride;
+            if (swap) { Dim t = d[a]; d[a] = d[bq]; d[bq] = t; }
+        }
+    // size-1 dimensions get a stride that keeps the list ascending
+    unsigned long long prev = (unsigned long long)kD * 2;
+    for (int a = 0; a < 3; ++a) {
+        if (d[a].size == 1 || d[a].stride < prev) d[a].stride = prev;
+        prev = d[a].stride * d[a].size;
+        slot[d[a].which] = a;
+    }
+    cuuint64_t gdim[4] = {(cuuint64_t)kD, d[0].size, d[1].size, d[2].size};
+    cuuint64_t gstr[3] = {d[0].stride, d[1].stride, d[2].stride};
+    cuuint32_t box[4] = {64, 1, 1, 1};
+    box[1 + slot[0]] = kBK;
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+}  // namespace
+
+bool tc_attention_shape_ok(const Call &c, int dtype) {
+    if (dtype != SLA_BF16 || c.D != kD) return false;
+    if (c.kv_st < kD || c.top_k > kMaxTopK) return false;
+    const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
+    const long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
+    return span_tokens / kBK + 2 <= 4096;
+}
+
+bool tc_attention_supported(const Call &c, int dtype) {
+    return tc_attention_shape_ok(c, dtype) && encode_fn() != nullptr;
+}
+
+// Scratch layout for a chunk of Lc query positions; returns total bytes.
+TcPlan plan_attention_tc(const Call &c, int Lc) {
+    TcPlan p;
+    p.Lc = Lc;
+    p.NB = (int)((c.Lkv + kBK - 1) / kBK);
+    const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
+    long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
+    if (span_tokens > c.Lkv) span_tokens = c.Lkv;
+    p.nb_max = (int)((span_tokens - 1) / kBK + 2);
+    p.n_groups = (long long)c.B * c.Hkv * p.NB;
+    p.n_keys = p.n_groups * p.nb_max;
+    const size_t rows = (size_t)c.B * c.Hq * Lc;
+    const size_t slots = rows * c.top_k;
+    p.max_tiles = (long long)(slots / kRows) + p.n_groups + 1;
+    size_t off = 0;
+    p.off_counters = off; off = align256(off + 64);
+    p.off_key_count = off; off = align256(off + (size_t)p.n_keys * 4);
+    p.off_key_cursor = off; off = align256(off + (size_t)p.n_keys * 4);
+    p.off_tiles = off; off = align256(off + (size_t)p.max_tiles * 16);
+    p.off_recs = off; off = align256(off + slots * 16);
+    p.off_npieces = off; off = align256(off + rows);
+    p.off_part_lse = off; off = align256(off + slots * 8);
+    p.off_part_o = off; off = align256(off + slots * kD * 2);
+    p.bytes = off;
+    return p;
+}
+
+cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor,
+                           void *out, float *lse, void *scratch, size_t scratch_bytes, int sm_count,
+                           cudaStream_t st, long long *launches) {
+    // the largest chunk of query positions whose scratch fits
+    long long Lc = c.Lq;
+    TcPlan plan = plan_attention_tc(c, (int)Lc);
+    while (plan.bytes > scratch_bytes && Lc > 1) {
+        Lc = (Lc + 1) / 2;
+        plan = plan_attention_tc(c, (int)Lc);
+    }
+    if (plan.bytes > scratch_bytes) return cudaErrorMemoryAllocation;
+    if (plan.n_keys > (1ll << 30) || (long long)c.B * c.Hq * Lc * c.top_k > (1ll << 31) - 1) return cudaErrorInvalidValue;
+
+    CUtensorMap tm_k, tm_v;
+    int slot[3];
+    if (!make_kv_map(&tm_k, k, c, slot) || !make_kv_map(&tm_v, v, c, slot)) return cudaErrorInvalidValue;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_attend, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    char *ws = (char *)scratch;
+    int *counters = (int *)(ws + plan.off_counters);
+    for (long long r0 = 0; r0 < c.Lq; r0 += Lc) {
+        const int lc = (int)((c.Lq - r0 < Lc) ? c.Lq - r0 : Lc);
+        const long long rows = (long long)c.B * c.Hq * lc;
+        cudaError_t e = cudaMemsetAsync(ws + plan.off_key_count, 0, plan.off_tiles - plan.off_key_count, st);
+        if (e != cudaSuccess) return e;
+        PrepParams pp;
+        pp.anchor = anchor; pp.B = c.B; pp.Hq = c.Hq; pp.Hkv = c.Hkv; pp.G = c.G; pp.top_k = c.top_k;
+        pp.span_len = c.span_len; pp.back = c.back; pp.fwd = c.fwd; pp.Lq = c.Lq; pp.q_pos0 = c.q_pos0;
+        pp.r0 = r0; pp.Lc = lc; pp.NB = plan.NB; pp.nb_max = plan.nb_max;
+        pp.key_count = (int *)(ws + plan.off_key_count);
+        pp.key_cursor = (int *)(ws + plan.off_key_cursor);
+        pp.recs = (int4 *)(ws + plan.off_recs);
+        pp.n_pieces = (unsigned char *)(ws + plan.off_npieces);
+        pp.status = c.status;
+        const unsigned blocks = (unsigned)((rows + 127) / 128);
+        tc_pieces<false><<<blocks, 128, 0, st>>>(pp);
+        tc_scan<<<1, 1024, 0, st>>>(pp.key_count, plan.n_keys, plan.nb_max, (int)plan.n_groups, plan.NB,
+                                    (int4 *)(ws + plan.off_tiles), counters, counters + 1, (int)plan.max_tiles);
+        tc_pieces<true><<<blocks, 128, 0, st>>>(pp);
+        TcParams tp;
+        tp.q = (const bf16 *)q; tp.q_sb = c.q_sb; tp.q_sh = c.q_sh; tp.q_st = c.q_st;
+        tp.Hq = c.Hq; tp.G = c.G; tp.Lc = lc; tp.top_k = c.top_k; tp.r0 = r0;
+        tp.scale2 = c.softmax_scale * kLog2e;
+        tp.slot_t = slot[0]; tp.slot_h = slot[1]; tp.slot_b = slot[2];
+        tp.recs = pp.recs; tp.tiles = (const int4 *)(ws + plan.off_tiles);
+        tp.n_tiles = counters; tp.tile_counter = counters + 1;
+        tp.part_o = (__half *)(ws + plan.off_part_o); tp.part_lse = (float2 *)(ws + plan.off_part_lse);
+        tp.status = c.status; tp.Hkv = c.Hkv;
+        tc_attend<<<2 * sm_count, kThreads, kSmemBytes, st>>>(tm_k, tm_v, tp);
+        const unsigned mblocks = (unsigned)((rows * 16 + 255) / 256);
+        tc_merge<<<mblocks, 256, 0, st>>>(tp.part_o, tp.part_lse, pp.n_pieces, c, lc, r0, (bf16 *)out, lse);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        if (launches) *launches += 5;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace sla

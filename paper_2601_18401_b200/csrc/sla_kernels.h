@@ -11,6 +11,23 @@ cudaError_t launch_search_simt(const void *q_s, const void *k, const Call &c, in
 cudaError_t launch_attn_simt(const void *q, const void *k, const void *v, const Call &c, int dtype,
                              const int32_t *anchor, void *out, float *lse, cudaStream_t st);
 
+// ---- tensor-core span-attention for prefill, bf16 / head_dim 128 (sla_attn_tc.cu) ---------------
+// Scratch layout for one chunk of Lc query positions (all offsets in bytes).
+struct TcPlan {
+    int Lc, NB, nb_max;
+    long long n_groups, n_keys, max_tiles;
+    size_t off_counters, off_key_count, off_key_cursor, off_tiles, off_recs, off_npieces, off_part_lse,
+        off_part_o, bytes;
+};
+bool tc_attention_shape_ok(const Call &c, int dtype);  // host-only shape test
+bool tc_attention_supported(const Call &c, int dtype); // shape test + driver entry point present
+TcPlan plan_attention_tc(const Call &c, int Lc);
+// Splits the query rows into chunks whose scratch fits `scratch_bytes`; adds its kernel launches to
+// *launches.  Returns cudaErrorMemoryAllocation when not even one query position fits.
+cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor,
+                           void *out, float *lse, void *scratch, size_t scratch_bytes, int sm_count,
+                           cudaStream_t st, long long *launches);
+
 // ---- decode step (sla_decode.cu) ---------------------------------------------------------------
 // Scratch layout of one decode step, all offsets in bytes from the scratch base.
 struct DecodePlan {
