@@ -30,6 +30,9 @@
 #include <cuda_fp16.h>
 #include <limits.h>
 #include <math_constants.h>
+#ifdef SLA_TC_TIMING
+#include <stdio.h>
+#endif
 
 #include "sla_kernels.h"
 #include "sla_tc_ptx.cuh"
@@ -49,23 +52,22 @@ constexpr uint32_t kColS = 0;    // S buffers at columns 0 and 64
 constexpr uint32_t kColO = 128;
 constexpr int kQBytes = kRows * kD * 2;      // 32 KiB, two 64-wide halves of 128 rows x 128 B
 constexpr int kKVBytes = kBK * kD * 2;       // 16 KiB, two 64-wide halves of 64 rows x 128 B
+constexpr int kKS = 3;           // K stages (a K block is free again as soon as its S = Q K^T is done)
+constexpr int kVS = 2;           // V stages (and S/P buffers)
 constexpr int kOffQ = 0;
 constexpr int kOffK = kQBytes;
-constexpr int kOffV = kOffK + 2 * kKVBytes;
-constexpr int kOffMeta = kOffV + 2 * kKVBytes;   // 98304
-constexpr int kMetaBytes = 2048;
-constexpr int kSmemBytes = kOffMeta + kMetaBytes + 1024;  // + slack for 1024-byte alignment
+constexpr int kOffV = kOffK + kKS * kKVBytes;
+constexpr int kOffMeta = kOffV + kVS * kKVBytes;   // 114688
+constexpr int kMetaBytes = 1024;
+// 113 KiB: two CTAs (plus 1 KiB of system reserve each) fill the 228 KiB of an SM exactly
+constexpr int kSmemBytes = kOffMeta + kMetaBytes;
 constexpr float kRescaleThreshold = 8.f;     // log2 units: P stays below 2^8
 
 struct Meta {
-    unsigned long long q_full, o_full;
-    unsigned long long kv_full[2], kv_empty[2], s_full[2], p_ready[2];
+    unsigned long long q_full, o_full, o_empty;
+    unsigned long long k_full[kKS], k_empty[kKS], v_full[kVS], v_empty[kVS], s_full[2], p_ready[2];
     uint32_t tmem_base;
-    int tile;
-    int sb_min;
     int abort_flag;
-    int lo[kRows];
-    int hi[kRows];
 };
 static_assert(sizeof(Meta) <= kMetaBytes, "meta block too large");
 
@@ -77,7 +79,7 @@ struct TcParams {
     float scale2;              // softmax_scale * log2(e)
     int slot_t, slot_h, slot_b;  // positions of (token, head, batch) among tensor-map coordinates 1..3
     const int4 *recs;          // sorted piece records {row, j, lo, hi}
-    const int4 *tiles;         // {b*Hkv+g, end block, first record, record count}
+    const int4 *tiles;         // {b*Hkv+g, end block, first record, record count | key blocks to walk << 8}
     const int *n_tiles;
     int *tile_counter;
     __half *part_o;            // [rows*top_k][128] normalised piece outputs, fp16 with one power-of-two
@@ -224,12 +226,15 @@ tc_scan(int *key_count, long long n_keys, int nb_max, int n_groups, int NB, int4
         const int nt = (cnt + kRows - 1) / kRows;
         int tot;
         const int off = block_excl_scan(nt, tot) + carry_s;
+        int cls = 0;   // class (blocks covered - 1) of the record the walk below has reached
         for (int t = 0; t < nt; ++t) {
             const int idx = off + t;
-            if (idx < max_tiles) {
-                const int left = cnt - t * kRows;
-                tiles[idx] = make_int4(g / NB, g % NB, first + t * kRows, left < kRows ? left : kRows);
-            }
+            const int left = cnt - t * kRows;
+            const int n_here = left < kRows ? left : kRows;
+            // records of a group are ordered by blocks covered, so the tile's last record covers most
+            const int last = first + t * kRows + n_here - 1;
+            while (cls + 1 < nb_max && key_count[(long long)g * nb_max + cls + 1] <= last) ++cls;
+            if (idx < max_tiles) tiles[idx] = make_int4(g / NB, g % NB, first + t * kRows, n_here | ((cls + 1) << 8));
         }
         __syncthreads();
         if (tid == 0) carry_s += tot;
@@ -242,7 +247,34 @@ tc_scan(int *key_count, long long n_keys, int nb_max, int n_groups, int NB, int4
 }
 
 // ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// packed fp32x2 arithmetic (two independent fp32 lanes per instruction)
+__device__ __forceinline__ unsigned long long pack2(float a, float b) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long r, float &a, float &b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r));
+}
+__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long fadd2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ float ex2_approx(float x) {
+#ifdef SLA_EXP_NOMUFU
+    return fmaf(x, 1e-3f, 1.f);
+#endif
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
@@ -250,24 +282,33 @@ __device__ __forceinline__ float ex2_approx(float x) {
 
 __global__ void __launch_bounds__(kThreads, 2)
 tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, TcParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = ptx::smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t *smem = smem_raw + (base - raw);
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t base = ptx::smem_u32(smem);
     Meta *meta = reinterpret_cast<Meta *>(smem + kOffMeta);
     volatile int *abort_flag = &meta->abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (base & 1023u) {   // the swizzled tiles need a 1024-byte aligned window: refuse rather than corrupt
+        if (tid == 0) atomicOr(p.status, kStatusTimeout);
+        return;
+    }
 
     const uint32_t bar_q_full = ptx::smem_u32(&meta->q_full), bar_o_full = ptx::smem_u32(&meta->o_full);
-    const uint32_t bar_kv_full = ptx::smem_u32(&meta->kv_full[0]), bar_kv_empty = ptx::smem_u32(&meta->kv_empty[0]);
+    const uint32_t bar_o_empty = ptx::smem_u32(&meta->o_empty);
+    const uint32_t bar_k_full = ptx::smem_u32(&meta->k_full[0]), bar_k_empty = ptx::smem_u32(&meta->k_empty[0]);
+    const uint32_t bar_v_full = ptx::smem_u32(&meta->v_full[0]), bar_v_empty = ptx::smem_u32(&meta->v_empty[0]);
     const uint32_t bar_s_full = ptx::smem_u32(&meta->s_full[0]), bar_p_ready = ptx::smem_u32(&meta->p_ready[0]);
 
     if (tid == 0) {
         ptx::mbar_init(bar_q_full, kRows);
         ptx::mbar_init(bar_o_full, 1);
+        ptx::mbar_init(bar_o_empty, 4);
+        for (int s = 0; s < kKS; ++s) {
+            ptx::mbar_init(bar_k_full + 8 * s, 1);
+            ptx::mbar_init(bar_k_empty + 8 * s, 1);
+        }
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar_kv_full + 8 * s, 1);
-            ptx::mbar_init(bar_kv_empty + 8 * s, 1);
+            ptx::mbar_init(bar_v_full + 8 * s, 1);
+            ptx::mbar_init(bar_v_empty + 8 * s, 1);
             ptx::mbar_init(bar_s_full + 8 * s, 1);
             ptx::mbar_init(bar_p_ready + 8 * s, kRows);
         }
@@ -290,122 +331,156 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
     constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(kRows, kBK, false, false);   // S = Q K^T, both K-major
     constexpr uint32_t kIdescO = ptx::idesc_bf16_f32(kRows, kD, false, true);     // O = P V, V is N-major
 
-    uint32_t n_kv = 0;    // key blocks processed so far by this CTA (stage / buffer = n & 1)
-    uint32_t n_tile = 0;  // tiles processed so far
+    // Tiles are dealt round-robin: CTA c takes tiles c, c + grid, c + 2 grid, ...  Every role reads its
+    // tile's table entry {b*Hkv+g, end block, first record, count | blocks << 8} straight from global
+    // memory, one tile ahead of where it is working, so nothing but mbarriers couples the roles.
+    const int n_tiles = *p.n_tiles;
+    const int tile_step = gridDim.x;
 
-    for (;;) {
-        __syncthreads();
-        if (tid == 0) {
-            int t = -1;
-            if (!*abort_flag) {
-                t = atomicAdd(p.tile_counter, 1);
-                if (t >= *p.n_tiles) t = -1;
-            }
-            meta->tile = t;
-            meta->sb_min = INT_MAX;
-        }
-        __syncthreads();
-        const int tile = meta->tile;
-        if (tile < 0) break;
-        const int4 ti = p.tiles[tile];   // {b*Hkv+g, end block, first record, count}
-
-        // ---- rows of the tile (warps 0-3, one row per thread)
-        int4 rec = make_int4(0, 0, INT_MAX, -1);
-        if (warp < 4) {
-            if (tid < ti.w) rec = p.recs[ti.z + tid];
-            meta->lo[tid] = rec.z;
-            meta->hi[tid] = rec.w;
-            int sb = tid < ti.w ? rec.z / kBK : INT_MAX;
-            sb = __reduce_min_sync(0xffffffffu, sb);
-            if (lane == 0) atomicMin(&meta->sb_min, sb);
-        }
-        __syncthreads();
-        const int sb0 = meta->sb_min;
-        const int nblk = ti.y - sb0 + 1;
-        const int g = ti.x % p.Hkv, b = ti.x / p.Hkv;
-
-        if (warp == 5) {
-            // ---------------- TMA producer
-            if (lane == 0) {
-                int c[4];
-                c[1 + p.slot_h] = g;
-                c[1 + p.slot_b] = b;
-                for (int j = 0; j < nblk; ++j) {
-                    const uint32_t n = n_kv + j, st = n & 1u, ph = (n >> 1) & 1u;
-                    if (!ptx::mbar_wait(bar_kv_empty + 8 * st, ph ^ 1u, abort_flag)) break;
-                    ptx::mbar_arrive_expect_tx(bar_kv_full + 8 * st, 2 * kKVBytes);
-                    c[1 + p.slot_t] = (sb0 + j) * kBK;
-                    const uint32_t dk = base + kOffK + st * kKVBytes, dv = base + kOffV + st * kKVBytes;
-                    ptx::tma_load_4d(dk, &tm_k, bar_kv_full + 8 * st, 0, c[1], c[2], c[3]);
-                    ptx::tma_load_4d(dk + kKVBytes / 2, &tm_k, bar_kv_full + 8 * st, 64, c[1], c[2], c[3]);
-                    ptx::tma_load_4d(dv, &tm_v, bar_kv_full + 8 * st, 0, c[1], c[2], c[3]);
-                    ptx::tma_load_4d(dv + kKVBytes / 2, &tm_v, bar_kv_full + 8 * st, 64, c[1], c[2], c[3]);
+    if (warp == 5 && lane == 0) {
+        // ---------------- TMA producer: K(j) then V(j) of every key block, as far ahead as the stages allow
+        uint32_t n_kv = 0;
+        int tile = blockIdx.x;
+        int4 ti = tile < n_tiles ? p.tiles[tile] : make_int4(0, 0, 0, 0);
+        for (; tile < n_tiles; tile += tile_step) {
+            const int nblk = ti.w >> 8, sb0 = ti.y - nblk + 1;
+            int c[4];
+            c[1 + p.slot_h] = ti.x % p.Hkv;
+            c[1 + p.slot_b] = ti.x / p.Hkv;
+            const int4 ti_next = tile + tile_step < n_tiles ? p.tiles[tile + tile_step] : make_int4(0, 0, 0, 0);
+            bool ok = true;
+            for (int j = 0; j < nblk; ++j) {
+                const uint32_t n = n_kv + j;
+                c[1 + p.slot_t] = (sb0 + j) * kBK;
+                {
+                    const uint32_t st = n % kKS, ph = (n / kKS) & 1u;
+                    ok = ptx::mbar_wait(bar_k_empty + 8 * st, ph ^ 1u, abort_flag);
+                    if (!ok) break;
+                    ptx::mbar_arrive_expect_tx(bar_k_full + 8 * st, kKVBytes);
+                    const uint32_t dst = base + kOffK + st * kKVBytes;
+                    ptx::tma_load_4d(dst, &tm_k, bar_k_full + 8 * st, 0, c[1], c[2], c[3]);
+                    ptx::tma_load_4d(dst + kKVBytes / 2, &tm_k, bar_k_full + 8 * st, 64, c[1], c[2], c[3]);
+                }
+                {
+                    const uint32_t st = n % kVS, ph = (n / kVS) & 1u;
+                    ok = ptx::mbar_wait(bar_v_empty + 8 * st, ph ^ 1u, abort_flag);
+                    if (!ok) break;
+                    ptx::mbar_arrive_expect_tx(bar_v_full + 8 * st, kKVBytes);
+                    const uint32_t dst = base + kOffV + st * kKVBytes;
+                    ptx::tma_load_4d(dst, &tm_v, bar_v_full + 8 * st, 0, c[1], c[2], c[3]);
+                    ptx::tma_load_4d(dst + kKVBytes / 2, &tm_v, bar_v_full + 8 * st, 64, c[1], c[2], c[3]);
                 }
             }
-        } else if (warp == 4) {
-            // ---------------- MMA issuer: S(0); S(1), PV(0); S(2), PV(1); ...
-            if (lane == 0) {
-                bool ok = ptx::mbar_wait(bar_q_full, n_tile & 1u, abort_flag);
-                ptx::tc_fence_after();
-                for (int step = 0; ok && step <= nblk; ++step) {
-                    if (step < nblk) {
-                        const uint32_t n = n_kv + step, st = n & 1u, ph = (n >> 1) & 1u;
-                        ok = ptx::mbar_wait(bar_kv_full + 8 * st, ph, abort_flag);
-                        if (!ok) break;
+            if (!ok) break;
+            n_kv += nblk;
+            ti = ti_next;
+        }
+    } else if (warp == 4 && lane == 0) {
+        // ---------------- MMA issuer, event driven: S(j) as soon as K(j) has landed and an S buffer
+        // is free, PV(j) as soon as P(j) and V(j) are there.  S(j+2) reuses the buffer of P(j), so it
+        // is only issued after PV(j); the first PV of a tile overwrites O, so it waits until the row
+        // threads have read the previous tile's O.
+        uint32_t n_kv = 0, T = 0;
+        int tile = blockIdx.x;
+        int nblk = tile < n_tiles ? (p.tiles[tile].w >> 8) : 0;
+        for (; tile < n_tiles; tile += tile_step, ++T) {
+            const int nblk_next = tile + tile_step < n_tiles ? (p.tiles[tile + tile_step].w >> 8) : 0;
+            bool ok = ptx::mbar_wait(bar_q_full, T & 1u, abort_flag);
+            ptx::tc_fence_after();
+            int is = 0, ipv = 0;
+            uint32_t idle = 0;
+            while (ok && ipv < nblk) {
+                bool progressed = false;
+                if (is < nblk && is < ipv + 2) {
+                    const uint32_t n = n_kv + is, ks = n % kKS, sbuf = n & 1u;
+                    if (ptx::mbar_test_wait(bar_k_full + 8 * ks, (n / kKS) & 1u)) {
                         ptx::tc_fence_after();
-                        const uint32_t d_s = tmem + kColS + st * kBK;
+                        const uint32_t d_s = tmem + kColS + sbuf * kBK;
 #pragma unroll
-                        for (int ks = 0; ks < kD / 16; ++ks) {
-                            const uint32_t half = ks >> 2, inner = (ks & 3) * 32;
+                        for (int kk = 0; kk < kD / 16; ++kk) {
+                            const uint32_t half = kk >> 2, inner = (kk & 3) * 32;
                             const uint64_t da = ptx::smem_desc_sw128(base + kOffQ + half * (kQBytes / 2) + inner, 16, 1024);
-                            const uint64_t db = ptx::smem_desc_sw128(base + kOffK + st * kKVBytes + half * (kKVBytes / 2) + inner, 16, 1024);
-                            ptx::mma_ss(d_s, da, db, kIdescS, ks > 0);
+                            const uint64_t db = ptx::smem_desc_sw128(base + kOffK + ks * kKVBytes + half * (kKVBytes / 2) + inner, 16, 1024);
+                            ptx::mma_ss(d_s, da, db, kIdescS, kk > 0);
                         }
-                        ptx::mma_commit(bar_s_full + 8 * st);
+                        ptx::mma_commit(bar_s_full + 8 * sbuf);
+                        ptx::mma_commit(bar_k_empty + 8 * ks);
+                        ++is;
+                        progressed = true;
                     }
-                    if (step >= 1) {
-                        const int jj = step - 1;
-                        const uint32_t n = n_kv + jj, st = n & 1u, ph = (n >> 1) & 1u;
-                        ok = ptx::mbar_wait(bar_p_ready + 8 * st, ph, abort_flag);
-                        if (!ok) break;
+                }
+                if (ipv < is) {
+                    const uint32_t n = n_kv + ipv, vs = n & 1u, ph = (n >> 1) & 1u;
+                    const bool o_free = ipv > 0 || T == 0 || ptx::mbar_test_wait(bar_o_empty, (T - 1u) & 1u);
+                    if (o_free && ptx::mbar_test_wait(bar_p_ready + 8 * vs, ph) && ptx::mbar_test_wait(bar_v_full + 8 * vs, ph)) {
                         ptx::tc_fence_after();
-                        const uint32_t a_p = tmem + kColS + st * kBK;   // P aliases S: 64 bf16 = 32 columns
+                        const uint32_t a_p = tmem + kColS + vs * kBK;   // P aliases S: 64 bf16 = 32 columns
 #pragma unroll
-                        for (int ks = 0; ks < kBK / 16; ++ks) {
-                            const uint64_t db = ptx::smem_desc_sw128(base + kOffV + st * kKVBytes + ks * 2048, kKVBytes / 2, 1024);
-                            ptx::mma_ts(tmem + kColO, a_p + ks * 8, db, kIdescO, (jj > 0 || ks > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < kBK / 16; ++kk) {
+                            const uint64_t db = ptx::smem_desc_sw128(base + kOffV + vs * kKVBytes + kk * 2048, kKVBytes / 2, 1024);
+                            ptx::mma_ts(tmem + kColO, a_p + kk * 8, db, kIdescO, (ipv > 0 || kk > 0) ? 1u : 0u);
                         }
-                        ptx::mma_commit(bar_kv_empty + 8 * st);
-                        if (jj == nblk - 1) ptx::mma_commit(bar_o_full);
+                        ptx::mma_commit(bar_v_empty + 8 * vs);
+                        if (ipv == nblk - 1) ptx::mma_commit(bar_o_full);
+                        ++ipv;
+                        progressed = true;
                     }
                 }
+                if (progressed) {
+                    idle = 0;
+                } else if (__nanosleep(20), ++idle > ptx::kSpinLimit || ((idle & 63u) == 0u && *abort_flag)) {
+                    *abort_flag = 1;
+                    ok = false;
+                }
             }
-        } else {
-            // ---------------- row threads: Q gather, softmax per key block, epilogue
-            const bool valid = tid < ti.w;
-            const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-            {
+            if (!ok) break;
+            n_kv += nblk;
+            nblk = nblk_next;
+        }
+    } else if (warp < 4) {
+        // ---------------- row threads: Q gather, softmax per key block, epilogue
+        const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+        const uint32_t q_row = base + kOffQ + tid * 128;
+        // Gathers one Q row (256 B) into the swizzled A-operand layout with 16-byte async copies.
+        auto gather_q = [&](bool row_valid, int row) {
+            if (row_valid) {
+                const int rc = row % p.Lc, bh = row / p.Lc;
+                const int h = bh % p.Hq, bb = bh / p.Hq;
+                const bf16 *src = p.q + bb * p.q_sb + h * p.q_sh + (p.r0 + rc) * p.q_st;
+#pragma unroll
+                for (int cidx = 0; cidx < 16; ++cidx) {
+                    const uint32_t dst = q_row + (cidx >> 3) * (kQBytes / 2) + (((cidx & 7) ^ (tid & 7)) << 4);
+                    ptx::cp_async16(dst, src + cidx * 8);
+                }
+            } else {
                 uint4 *qdst = reinterpret_cast<uint4 *>(smem + kOffQ);
-                if (valid) {
-                    const int rc = rec.x % p.Lc, bh = rec.x / p.Lc;
-                    const int h = bh % p.Hq, bb = bh / p.Hq;
-                    const uint4 *src = reinterpret_cast<const uint4 *>(p.q + bb * p.q_sb + h * p.q_sh + (p.r0 + rc) * p.q_st);
-                    uint4 v[16];
 #pragma unroll
-                    for (int cidx = 0; cidx < 16; ++cidx) v[cidx] = __ldg(src + cidx);
-#pragma unroll
-                    for (int cidx = 0; cidx < 16; ++cidx) {
-                        const int half = cidx >> 3, ch = (cidx & 7) ^ (tid & 7);
-                        qdst[half * (kQBytes / 32) + tid * 8 + ch] = v[cidx];
-                    }
-                } else {
-#pragma unroll
-                    for (int cidx = 0; cidx < 16; ++cidx)
-                        qdst[(cidx >> 3) * (kQBytes / 32) + tid * 8 + (cidx & 7)] = make_uint4(0, 0, 0, 0);
-                }
-                ptx::fence_proxy_async_smem();
-                ptx::mbar_arrive(bar_q_full);
+                for (int cidx = 0; cidx < 16; ++cidx)
+                    qdst[(cidx >> 3) * (kQBytes / 32) + tid * 8 + (cidx & 7)] = make_uint4(0, 0, 0, 0);
             }
+        };
+        uint32_t n_kv = 0, T = 0;
+        int tile = blockIdx.x;
+        int4 ti = tile < n_tiles ? p.tiles[tile] : make_int4(0, 0, 0, 0);
+        int4 rec = make_int4(0, 0, INT_MAX, -1);
+        if (tile < n_tiles) {
+            if (tid < (ti.w & 0xff)) rec = p.recs[ti.z + tid];
+            gather_q(tid < (ti.w & 0xff), rec.x);
+        }
+        for (; tile < n_tiles; tile += tile_step, ++T) {
+            const int nblk = ti.w >> 8, sb0 = ti.y - nblk + 1, cnt = ti.w & 0xff;
+            const bool valid = tid < cnt;
+            // hand this tile's Q to the MMA issuer
+            ptx::cp_async_wait_all();
+            ptx::fence_proxy_async_smem();
+            ptx::mbar_arrive(bar_q_full);
+            // the next tile: its record is fetched now, its Q row during this tile's last key block
+            const bool has_next = tile + tile_step < n_tiles;
+            const int4 ti_next = has_next ? p.tiles[tile + tile_step] : make_int4(0, 0, 0, 0);
+            const int cnt_next = ti_next.w & 0xff;
+            int4 rec_next = make_int4(0, 0, INT_MAX, -1);
+            if (has_next && tid < cnt_next) rec_next = p.recs[ti_next.z + tid];
+
             const int lo = rec.z, hi = rec.w;
             float m_ref = -CUDART_INF_F, l = 0.f;
             bool ok = true;
@@ -414,6 +489,8 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 ok = ptx::mbar_wait_warp(bar_s_full + 8 * st, ph, abort_flag);
                 if (!ok) break;
                 ptx::tc_fence_after();
+                // S of the last block is done, so nothing reads this tile's Q any more
+                if (j == nblk - 1 && has_next) gather_q(tid < cnt_next, rec_next.x);
                 const uint32_t s_addr = lane_addr + kColS + st * kBK;
                 uint32_t sr[2][32];
                 ptx::tmem_ld32(s_addr, sr[0]);
@@ -422,20 +499,27 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 const int k0 = (sb0 + j) * kBK;
                 const bool any = valid && k0 <= hi && k0 + kBK - 1 >= lo;
                 const bool full = any && k0 >= lo && k0 + kBK - 1 <= hi;
+                // block maximum on the raw logits (softmax_scale > 0 on this path), four independent chains
                 float bm = -CUDART_INF_F;
                 if (any) {
+                    if (!full) {
+#pragma unroll
+                        for (int hlf = 0; hlf < 2; ++hlf)
+#pragma unroll
+                            for (int cc = 0; cc < 32; ++cc) {
+                                const int kp = k0 + hlf * 32 + cc;
+                                if (kp < lo || kp > hi) sr[hlf][cc] = 0xff800000u;   // -inf
+                            }
+                    }
+                    float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
                     for (int hlf = 0; hlf < 2; ++hlf)
 #pragma unroll
-                        for (int cc = 0; cc < 32; ++cc) {
-                            float x = __uint_as_float(sr[hlf][cc]) * p.scale2;
-                            if (!full) {
-                                const int kp = k0 + hlf * 32 + cc;
-                                x = (kp >= lo && kp <= hi) ? x : -CUDART_INF_F;
-                            }
-                            sr[hlf][cc] = __float_as_uint(x);
-                            bm = fmaxf(bm, x);
-                        }
+                        for (int cc = 0; cc < 32; cc += 8)
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                mx[u] = max3(mx[u], __uint_as_float(sr[hlf][cc + 2 * u]), __uint_as_float(sr[hlf][cc + 2 * u + 1]));
+                    bm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale2;
                 }
                 // running reference maximum; O is rescaled only when it moves by more than the threshold
                 const bool first = (l == 0.f);   // no key of this row seen so far
@@ -443,7 +527,7 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 if (__any_sync(0xffffffffu, need)) {
                     // PV of the previous block must have landed before O is touched
                     const uint32_t np = n - 1u;
-                    ok = ptx::mbar_wait_warp(bar_kv_empty + 8 * (np & 1u), (np >> 1) & 1u, abort_flag);
+                    ok = ptx::mbar_wait_warp(bar_v_empty + 8 * (np & 1u), (np >> 1) & 1u, abort_flag);
                     if (!ok) break;
                     ptx::tc_fence_after();
                     const float f = need ? ex2_approx(m_ref - bm) : 1.f;
@@ -461,17 +545,27 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 if (first && bm > -CUDART_INF_F) m_ref = bm;   // first keys of this row
                 uint32_t pk[32];
                 if (any && bm > -CUDART_INF_F) {
-                    float sum = 0.f;
+                    // p = 2^(s*scale - m_ref), two columns per packed fp32x2 instruction
+                    const unsigned long long sc2 = pack2(p.scale2, p.scale2), nm2 = pack2(-m_ref, -m_ref);
+                    unsigned long long acc2[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) acc2[u] = pack2(0.f, 0.f);
 #pragma unroll
                     for (int cc = 0; cc < 32; ++cc) {
                         const int hlf = cc >> 4, c2 = (cc & 15) * 2;
-                        const float p0 = ex2_approx(__uint_as_float(sr[hlf][c2]) - m_ref);
-                        const float p1 = ex2_approx(__uint_as_float(sr[hlf][c2 + 1]) - m_ref);
-                        sum += p0 + p1;
+                        const unsigned long long y = ffma2(
+                            pack2(__uint_as_float(sr[hlf][c2]), __uint_as_float(sr[hlf][c2 + 1])), sc2, nm2);
+                        float y0, y1;
+                        unpack2(y, y0, y1);
+                        const float p0 = ex2_approx(y0), p1 = ex2_approx(y1);
+                        acc2[cc & 3] = fadd2(acc2[cc & 3], pack2(p0, p1));
                         const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
                         pk[cc] = *reinterpret_cast<const uint32_t *>(&pp);
                     }
-                    l += sum;
+                    float s0, s1, s2, s3;
+                    unpack2(fadd2(acc2[0], acc2[1]), s0, s1);
+                    unpack2(fadd2(acc2[2], acc2[3]), s2, s3);
+                    l += (s0 + s1) + (s2 + s3);
                 } else {
 #pragma unroll
                     for (int cc = 0; cc < 32; ++cc) pk[cc] = 0u;
@@ -482,12 +576,13 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 ptx::mbar_arrive(bar_p_ready + 8 * st);
             }
             // epilogue: normalised piece output and its log-sum-exp
-            if (ok) ok = ptx::mbar_wait_warp(bar_o_full, n_tile & 1u, abort_flag);
-            if (ok) {
-                ptx::tc_fence_after();
+            if (ok) ok = ptx::mbar_wait_warp(bar_o_full, T & 1u, abort_flag);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            {
                 const float inv = l > 0.f ? 1.f / l : 0.f;
                 const long long slot = (long long)rec.x * p.top_k + rec.y;
-                uint4 *dst = reinterpret_cast<uint4 *>(p.part_o + slot * kD);
+                __half *dst = p.part_o + slot * kD;
                 uint32_t exps = 0;   // biased exponent of each 32-column chunk's largest magnitude
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
@@ -507,25 +602,30 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                         exps |= eb << (8 * q4);
                         const float down = __uint_as_float((253u - eb) << 23);   // 2^(126 - eb): chunk into [-1, 1]
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
-                            uint32_t w[4];
+                        for (int s8 = 0; s8 < 2; ++s8) {
+                            uint32_t w[8];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const __half2 pp = __floats2half2_rn(__uint_as_float(o[v4 * 8 + 2 * e]) * down,
-                                                                     __uint_as_float(o[v4 * 8 + 2 * e + 1]) * down);
+                            for (int e = 0; e < 8; ++e) {
+                                const __half2 pp = __floats2half2_rn(__uint_as_float(o[s8 * 16 + 2 * e]) * down,
+                                                                     __uint_as_float(o[s8 * 16 + 2 * e + 1]) * down);
                                 w[e] = *reinterpret_cast<const uint32_t *>(&pp);
                             }
-                            dst[q4 * 4 + v4] = make_uint4(w[0], w[1], w[2], w[3]);
+                            ptx::st_global_v8(dst + q4 * 32 + s8 * 16, w);
                         }
                     }
                 }
                 if (valid)
                     p.part_lse[slot] = make_float2(l > 0.f ? m_ref + log2f(l) : -CUDART_INF_F, __uint_as_float(exps));
-                ptx::tc_fence_before();
             }
+            // O has been read: the next tile's first PV may overwrite it
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar_o_empty);
+            n_kv += nblk;
+            rec = rec_next;
+            ti = ti_next;
         }
-        n_kv += nblk;
-        n_tile += 1;
+        ptx::cp_async_wait_all();
     }
 
     // ---- teardown
@@ -648,7 +748,7 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 bool tc_attention_shape_ok(const Call &c, int dtype) {
     if (dtype != SLA_BF16 || c.D != kD) return false;
-    if (c.kv_st < kD || c.top_k > kMaxTopK) return false;
+    if (c.kv_st < kD || c.top_k > kMaxTopK || !(c.softmax_scale > 0.f)) return false;
     const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
     const long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     return span_tokens / kBK + 2 <= 4096;
