@@ -181,8 +181,13 @@ sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int
     if (!aligned16(q_s) || !aligned16(k)) return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
     if (sla_status_t s = check_supported(h, p)) return s;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
-    cudaError_t e = sla::launch_search_simt(q_s, k, c, l->dtype, out_anchor, out_score,
-                                            static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!h->force_simt && sla::search_mma_supported(c, l->dtype)) {
+        cudaError_t e = sla::launch_search_mma(q_s, k, c, out_anchor, out_score, st, &h->launches);
+        if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_search (tensor-core path)");
+        return SLA_OK;
+    }
+    cudaError_t e = sla::launch_search_simt(q_s, k, c, l->dtype, out_anchor, out_score, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_search");
     h->launches += 1;
     return SLA_OK;

@@ -11,6 +11,11 @@ cudaError_t launch_search_simt(const void *q_s, const void *k, const Call &c, in
 cudaError_t launch_attn_simt(const void *q, const void *k, const void *v, const Call &c, int dtype,
                              const int32_t *anchor, void *out, float *lse, cudaStream_t st);
 
+// ---- tensor-core span-search for bf16 / head_dim 128 (sla_search_mma.cu) -------------------------
+bool search_mma_supported(const Call &c, int dtype);
+cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int32_t *out_anchor, float *out_score,
+                              cudaStream_t st, long long *launches);
+
 // ---- tensor-core span-attention for prefill, bf16 / head_dim 128 (sla_attn_tc.cu) ---------------
 // Scratch layout for one chunk of Lc query positions (all offsets in bytes).
 struct TcPlan {

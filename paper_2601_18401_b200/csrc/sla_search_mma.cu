@@ -1,0 +1,215 @@
+// Span-search for bf16, head_dim 128 (Section "Span search": s_{i,t} = <Q_s(i), K(t)> over the
+// anchors t_s = i + 1 - (s+1)^2, then TopK).
+//
+// One warp owns one (batch, KV head, query position) and scores the anchors for all G query heads
+// of the group at once: 16 anchors x 128 dims of gathered K rows are the A operand of eight
+// m16n8k16 tensor-core MMAs, the group's routing queries (up to 8 heads) are the B operand, so every
+// K row is fetched once per group.  The work is a skinny gathered product (N = G <= 8) bound by the
+// L2 -> SM traffic of the key rows, not a dense contraction, which is why it runs on register-level
+// MMAs fed by plain 16-byte loads and not on tcgen05 tiles.  The dims are assigned to the MMA's k
+// slots in a permuted order (identical for A and B, which leaves the dot product unchanged) so that
+// each lane loads 16 contiguous bytes of a row.
+//
+// Scores go to shared memory; the k best of each head are then selected with warp votes: a
+// threshold from the lanes' maxima, compaction of the candidates above it, and k rounds of a
+// warp-wide arg-max (largest score first, smaller stride index on ties).
+#include <limits.h>
+#include <math_constants.h>
+
+#include "sla_kernels.h"
+
+namespace sla {
+
+namespace {
+
+using bf16 = __nv_bfloat16;
+constexpr int kWarps = 8;
+constexpr int kCap = 64;   // candidate slots per warp in the selection
+
+__device__ __forceinline__ uint32_t order_key(float x) {
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Top-k of sc[0..n) for one head; writes anchors/scores.  All lanes of the warp take part.
+__device__ void select_topk(float *sc, int n, int top_k, long long i, float *cand_v, int *cand_s,
+                            int32_t *out_anchor, float *out_score, int lane) {
+    const uint32_t kNegInfKey = order_key(-CUDART_INF_F);
+    // A. lane maxima over the strided slots
+    float lm = -CUDART_INF_F;
+    for (int s = lane; s < n; s += 32) lm = fmaxf(lm, sc[s]);
+    // B. threshold = top_k-th largest lane maximum (there are at least top_k scores >= it)
+    uint32_t cur = order_key(lm), tau_key = kNegInfKey;
+    if (n > top_k && top_k <= 32) {
+        for (int j = 0; j < top_k; ++j) {
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, cur);
+            tau_key = mx;
+            if (mx == kNegInfKey) break;
+            const uint32_t who = __ballot_sync(0xffffffffu, cur == mx);
+            if (lane == __ffs(who) - 1) cur = kNegInfKey;
+        }
+    }
+    // C. compact the candidates >= threshold
+    int count = 0;
+    for (int s0 = 0; s0 < n; s0 += 32) {
+        const int s = s0 + lane;
+        const float v = s < n ? sc[s] : 0.f;
+        const bool take = s < n && order_key(v) >= tau_key;
+        const uint32_t mask = __ballot_sync(0xffffffffu, take);
+        if (take) {
+            const int pos = count + __popc(mask & ((1u << lane) - 1u));
+            if (pos < kCap) { cand_v[pos] = v; cand_s[pos] = s; }
+        }
+        count += __popc(mask);
+    }
+    __syncwarp();
+    if (count <= kCap) {
+        // D. k rounds of warp arg-max over the candidates (two per lane)
+        float v0 = lane < count ? cand_v[lane] : -CUDART_INF_F, v1 = lane + 32 < count ? cand_v[lane + 32] : -CUDART_INF_F;
+        int s0 = lane < count ? cand_s[lane] : INT_MAX, s1 = lane + 32 < count ? cand_s[lane + 32] : INT_MAX;
+        for (int j = 0; j < top_k; ++j) {
+            const bool first = v0 > v1 || (v0 == v1 && s0 <= s1);
+            const float bv = first ? v0 : v1;
+            const int bs = first ? s0 : s1;
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, order_key(bv));
+            const int smin = __reduce_min_sync(0xffffffffu, (order_key(bv) == mx && bs != INT_MAX) ? bs : INT_MAX);
+            if (smin == INT_MAX) {   // fewer candidates than slots: pad
+                if (lane == 0) { out_anchor[j] = -1; out_score[j] = -CUDART_INF_F; }
+                continue;
+            }
+            if (bs == smin && order_key(bv) == mx) {
+                out_anchor[j] = (int32_t)(i + 1 - (long long)(bs + 1) * (bs + 1));
+                out_score[j] = bv;
+                if (first) { v0 = -CUDART_INF_F; s0 = INT_MAX; } else { v1 = -CUDART_INF_F; s1 = INT_MAX; }
+            }
+        }
+    } else {
+        // many equal scores at the threshold: plain k rounds over all scores
+        for (int j = 0; j < top_k; ++j) {
+            float bv = -CUDART_INF_F;
+            int bs = INT_MAX;
+            for (int s = lane; s < n; s += 32) {
+                const float v = sc[s];
+                if (v > bv) { bv = v; bs = s; }
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                const int os = __shfl_xor_sync(0xffffffffu, bs, off);
+                if (ov > bv || (ov == bv && os < bs)) { bv = ov; bs = os; }
+            }
+            if (lane == 0) {
+                if (bs != INT_MAX) {
+                    out_anchor[j] = (int32_t)(i + 1 - (long long)(bs + 1) * (bs + 1));
+                    out_score[j] = bv;
+                    sc[bs] = -CUDART_INF_F;
+                } else {
+                    out_anchor[j] = -1;
+                    out_score[j] = -CUDART_INF_F;
+                }
+            }
+            __syncwarp();
+        }
+    }
+    __syncwarp();
+}
+
+__global__ void __launch_bounds__(kWarps * 32)
+search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int32_t *__restrict__ out_anchor,
+           float *__restrict__ out_score, int n_max, int head0, int heads) {
+    extern __shared__ float smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long gid = (long long)blockIdx.x * kWarps + warp;   // (b, g, r)
+    if (gid >= (long long)c.B * c.Hkv * c.Lq) return;
+    const long long r = gid % c.Lq;
+    const int bg = (int)(gid / c.Lq), g = bg % c.Hkv, b = bg / c.Hkv;
+    const long long i = c.q_pos0 + r;
+    const int n = (int)isqrt_ll(i + 1);
+    float *sc = smem + (size_t)warp * (heads * n_max + 2 * kCap);
+    float *cand_v = sc + heads * n_max;
+    int *cand_s = reinterpret_cast<int *>(cand_v + kCap);
+
+    const int r8 = lane >> 2, q = lane & 3;
+    // B operand: routing queries of heads head0 .. head0+heads-1 of the group (column r8 of the MMA)
+    uint32_t bq[4][4];
+    {
+        const bool hv = r8 < heads;
+        const bf16 *qrow = q_s + b * c.q_sb + (long long)(g * c.G + head0 + (hv ? r8 : 0)) * c.q_sh + r * c.q_st;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (hv) v = __ldg(reinterpret_cast<const uint4 *>(qrow + 32 * ch + 8 * q));
+            bq[ch][0] = v.x; bq[ch][1] = v.y; bq[ch][2] = v.z; bq[ch][3] = v.w;
+        }
+    }
+    const bf16 *kbase = k + b * c.kv_sb + g * c.kv_sh + 8 * q;
+    for (int a0 = 0; a0 < n; a0 += 16) {
+        const int s0 = a0 + r8, s1 = s0 + 8;
+        const long long t0 = s0 < n ? i + 1 - (long long)(s0 + 1) * (s0 + 1) : i;
+        const long long t1 = s1 < n ? i + 1 - (long long)(s1 + 1) * (s1 + 1) : i;
+        uint4 ra[4], rb[4];
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            ra[ch] = __ldg(reinterpret_cast<const uint4 *>(kbase + t0 * c.kv_st + 32 * ch));
+            rb[ch] = __ldg(reinterpret_cast<const uint4 *>(kbase + t1 * c.kv_st + 32 * ch));
+        }
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            mma_bf16_16816(acc, ra[ch].x, rb[ch].x, ra[ch].y, rb[ch].y, bq[ch][0], bq[ch][1]);
+            mma_bf16_16816(acc, ra[ch].z, rb[ch].z, ra[ch].w, rb[ch].w, bq[ch][2], bq[ch][3]);
+        }
+        // acc[0],acc[1]: anchor s0, heads 2q, 2q+1;  acc[2],acc[3]: anchor s1
+        if (2 * q < heads) {
+            if (s0 < n) sc[(2 * q) * n_max + s0] = acc[0] * c.search_scale;
+            if (s1 < n) sc[(2 * q) * n_max + s1] = acc[2] * c.search_scale;
+        }
+        if (2 * q + 1 < heads) {
+            if (s0 < n) sc[(2 * q + 1) * n_max + s0] = acc[1] * c.search_scale;
+            if (s1 < n) sc[(2 * q + 1) * n_max + s1] = acc[3] * c.search_scale;
+        }
+    }
+    __syncwarp();
+    for (int hh = 0; hh < heads; ++hh) {
+        const int h = g * c.G + head0 + hh;
+        const long long obase = ((((long long)b * c.Hq + h) * c.Lq) + r) * c.top_k;
+        select_topk(sc + hh * n_max, n, c.top_k, i, cand_v, cand_s, out_anchor + obase, out_score + obase, lane);
+    }
+}
+
+}  // namespace
+
+bool search_mma_supported(const Call &c, int dtype) {
+    if (dtype != SLA_BF16 || c.D != 128) return false;
+    const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
+    const int heads = c.G < 8 ? c.G : 8;
+    return (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float) <= 200 * 1024;
+}
+
+cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int32_t *oa, float *os, cudaStream_t st,
+                              long long *launches) {
+    const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
+    const long long groups = (long long)c.B * c.Hkv * c.Lq;
+    const unsigned blocks = (unsigned)((groups + kWarps - 1) / kWarps);
+    for (int head0 = 0; head0 < c.G; head0 += 8) {
+        const int heads = c.G - head0 < 8 ? c.G - head0 : 8;
+        const size_t smem = (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float);
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(search_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        search_mma<<<blocks, kWarps * 32, smem, st>>>((const bf16 *)q_s, (const bf16 *)k, c, oa, os, n_max, head0, heads);
+        if (launches) *launches += 1;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace sla
