@@ -208,7 +208,8 @@ sla_status_t sla_span_attention(sla_handle_t h, const void *q, const void *k, co
     if (!h->force_simt && sla::tc_attention_supported(c, l->dtype)) {
         // tensor-core path; needs scratch for at least a modest chunk of query positions
         const long long min_chunk = Lq < 1024 ? Lq : 1024;
-        if (sla::plan_attention_tc(c, (int)min_chunk).bytes <= h->scratch_avail) {
+        const sla::TcPlan probe = sla::plan_attention_tc(c, (int)min_chunk);
+        if (probe.ok && probe.bytes <= h->scratch_avail) {
             cudaError_t e = sla::launch_attn_tc(q, k, v, c, anchor, out, lse, h->ws + kHeaderBytes,
                                                 h->scratch_avail, h->sm_count, st, &h->launches);
             if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_attention (tensor-core path)");

@@ -1,0 +1,224 @@
+// Work-list construction for the tensor-core span-attention kernel: a counting sort of all pieces
+// (clipped spans) of a chunk of query rows by (batch*Hkv + kv head, 64-key block of the piece's
+// right end, class of blocks covered), and the table of 128-piece tiles cut from the sorted list.
+//
+// This is the step Section "Kernel design" describes as grouping (query, span) pairs into buckets by
+// key-block footprint without a global sort.  Each CTA owns a slice of the rows of one
+// (batch, kv head), counts its pieces in a shared-memory histogram and touches the global counters
+// once per non-empty bucket, so that global atomics stay far below one per piece.
+//
+//   prep_pieces<0>   histogram of bucket sizes (+ number of pieces of every row)
+//   prep_scan_local  per (batch, kv head): exclusive offsets of its buckets, record and tile totals
+//   prep_scan_global per (batch, kv head): global offsets, tile table entries
+//   prep_pieces<1>   piece records to their places
+//   prep_tile_bounds per tile: how far back its pieces reach (number of key blocks to walk)
+#include <limits.h>
+
+#include "sla_attn_tc.cuh"
+
+namespace sla {
+namespace tc {
+
+namespace {
+
+constexpr int kPrepThreads = 1024;
+
+__device__ __forceinline__ int bucket_of(int lo, int hi, int ncls, int nb_max) {
+    const int eb = hi / kBK, sb = lo / kBK;
+    int cls = ((eb - sb) * ncls) / nb_max;
+    cls = cls < ncls ? cls : ncls - 1;
+    return eb * ncls + cls;
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
+    extern __shared__ int hist[];   // [NB * ncls]
+    const int nk = a.NB * a.ncls;
+    const int bg = blockIdx.x / a.ctas_per_bg, part = blockIdx.x % a.ctas_per_bg;
+    const int g = bg % a.Hkv, b = bg / a.Hkv;
+    const long long rows_bg = (long long)a.G * a.Lc;
+    const long long per = (rows_bg + a.ctas_per_bg - 1) / a.ctas_per_bg;
+    const long long q0 = per * part, q1 = (q0 + per < rows_bg) ? q0 + per : rows_bg;
+    int *gcount = a.key_count + (long long)bg * nk;
+    int *gcursor = a.key_cursor + (long long)bg * nk;
+    for (int x = threadIdx.x; x < nk; x += kPrepThreads) hist[x] = 0;
+    __syncthreads();
+
+    int lo[kMaxTopK], hi[kMaxTopK];
+    // sub-pass A: this CTA's pieces per bucket
+    for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
+        const int hg = (int)(q / a.Lc), rc = (int)(q % a.Lc);
+        const int h = g * a.G + hg;
+        const long long r = a.r0 + rc, i = a.q_pos0 + r;
+        const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
+        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len), a.back, a.fwd, lo, hi, a.status);
+        if (PASS == 0) a.n_pieces[((long long)b * a.Hq + h) * a.Lc + rc] = (unsigned char)cnt;
+        for (int j = 0; j < cnt; ++j) atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+    }
+    __syncthreads();
+    if constexpr (PASS == 0) {
+        for (int x = threadIdx.x; x < nk; x += kPrepThreads)
+            if (hist[x]) atomicAdd(gcount + x, hist[x]);
+    } else {
+    // claim a contiguous range of every non-empty bucket for this CTA
+    for (int x = threadIdx.x; x < nk; x += kPrepThreads) {
+        const int cnt = hist[x];
+        hist[x] = cnt ? gcount[x] + atomicAdd(gcursor + x, cnt) : 0;
+    }
+    __syncthreads();
+    // sub-pass B: write the records
+    for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
+        const int hg = (int)(q / a.Lc), rc = (int)(q % a.Lc);
+        const int h = g * a.G + hg;
+        const long long r = a.r0 + rc, i = a.q_pos0 + r;
+        const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
+        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len), a.back, a.fwd, lo, hi, a.status);
+        const int row = (int)(((long long)b * a.Hq + h) * a.Lc + rc);
+        for (int j = 0; j < cnt; ++j) {
+            const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+            a.recs[pos] = make_int4(row, j, lo[j], hi[j]);
+        }
+    }
+    }
+}
+
+// Exclusive scan over the block: returns this thread's offset, total in `total`.
+__device__ inline int block_excl_scan(int v, int &total, int *warp_sum) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int x = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, x, off);
+        if (lane >= off) x += y;
+    }
+    if (lane == 31) warp_sum[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_sum[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, w, off);
+            if (lane >= off) w += y;
+        }
+        warp_sum[lane] = w;
+    }
+    __syncthreads();
+    total = warp_sum[31];
+    const int base = warp > 0 ? warp_sum[warp - 1] : 0;
+    __syncthreads();
+    return base + x - v;
+}
+
+// One CTA per (batch, kv head): bucket histogram -> exclusive offsets local to the (batch, kv head),
+// plus how many records and tiles it has.
+__global__ void __launch_bounds__(kPrepThreads) prep_scan_local(PrepArgs a) {
+    __shared__ int warp_sum[32];
+    const int nk = a.NB * a.ncls, bg = blockIdx.x, tid = threadIdx.x;
+    int *cnt = a.key_count + (long long)bg * nk;
+    const int per = (nk + kPrepThreads - 1) / kPrepThreads;
+    const int k0 = per * tid, k1 = (k0 + per < nk) ? k0 + per : nk;
+    int local = 0;
+    for (int k = k0; k < k1; ++k) local += cnt[k];
+    int n_recs;
+    int run = block_excl_scan(local, n_recs, warp_sum);
+    for (int k = k0; k < k1; ++k) {
+        const int c = cnt[k];
+        cnt[k] = run;
+        run += c;
+    }
+    __syncthreads();
+    // tiles: every group (end block) is cut into tiles of kRows records
+    int tiles_local = 0;
+    for (int eb = tid; eb < a.NB; eb += kPrepThreads) {
+        const int first = cnt[eb * a.ncls];
+        const int last = (eb + 1 < a.NB) ? cnt[(eb + 1) * a.ncls] : n_recs;
+        tiles_local += (last - first + kRows - 1) / kRows;
+    }
+    int n_tiles;
+    block_excl_scan(tiles_local, n_tiles, warp_sum);
+    if (tid == 0) {
+        a.totals[2 * bg] = n_recs;
+        a.totals[2 * bg + 1] = n_tiles;
+    }
+}
+
+// One CTA per (batch, kv head): offsets become global, tile table entries are written.
+__global__ void __launch_bounds__(kPrepThreads) prep_scan_global(PrepArgs a) {
+    __shared__ int warp_sum[32];
+    __shared__ int s_base[2];
+    const int nk = a.NB * a.ncls, bg = blockIdx.x, tid = threadIdx.x, n_bg = a.B * a.Hkv;
+    if (tid == 0) {
+        int rec_base = 0, tile_base = 0;
+        for (int x = 0; x < bg; ++x) { rec_base += a.totals[2 * x]; tile_base += a.totals[2 * x + 1]; }
+        s_base[0] = rec_base;
+        s_base[1] = tile_base;
+        if (bg == n_bg - 1) {
+            const int all = tile_base + a.totals[2 * bg + 1];
+            *a.n_tiles = all < a.max_tiles ? all : a.max_tiles;
+        }
+    }
+    __syncthreads();
+    const int rec_base = s_base[0], tile_base = s_base[1], n_recs = a.totals[2 * bg];
+    int *cnt = a.key_count + (long long)bg * nk;
+    // tile entries first (they read the local offsets), in rounds of kPrepThreads groups
+    int carry = 0;
+    for (int eb0 = 0; eb0 < a.NB; eb0 += kPrepThreads) {
+        const int eb = eb0 + tid;
+        int first = 0, n = 0;
+        if (eb < a.NB) {
+            first = cnt[eb * a.ncls];
+            n = ((eb + 1 < a.NB) ? cnt[(eb + 1) * a.ncls] : n_recs) - first;
+        }
+        const int nt = (n + kRows - 1) / kRows;
+        int tot;
+        const int off = block_excl_scan(nt, tot, warp_sum) + carry + tile_base;
+        for (int t = 0; t < nt; ++t) {
+            const int left = n - t * kRows;
+            if (off + t < a.max_tiles)
+                a.tiles[off + t] = make_int4(bg, eb, rec_base + first + t * kRows, left < kRows ? left : kRows);
+        }
+        carry += tot;
+    }
+    __syncthreads();
+    for (int k = tid; k < nk; k += kPrepThreads) cnt[k] += rec_base;
+}
+
+// One warp per tile: the tile walks the key blocks from the one its furthest-reaching piece starts
+// in up to its end block; the count goes into bits 8.. of the entry's last word.
+__global__ void __launch_bounds__(256) prep_tile_bounds(PrepArgs a) {
+    const int t = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (t >= *a.n_tiles) return;
+    int4 ti = a.tiles[t];
+    int lo = INT_MAX;
+    for (int x = lane; x < ti.w; x += 32) lo = min(lo, a.recs[ti.z + x].z);
+    lo = __reduce_min_sync(0xffffffffu, lo);
+    if (lane == 0) {
+        ti.w |= (ti.y - lo / kBK + 1) << 8;
+        a.tiles[t] = ti;
+    }
+}
+
+}  // namespace
+
+cudaError_t prepare(const PrepArgs &a, cudaStream_t st, long long *launches) {
+    const int n_bg = a.B * a.Hkv;
+    const size_t smem = (size_t)a.NB * a.ncls * sizeof(int);
+    static size_t attr_bytes = 0;
+    if (smem > 48 * 1024 && smem > attr_bytes) {
+        cudaError_t e = cudaFuncSetAttribute(prep_pieces<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(prep_pieces<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_bytes = smem;
+    }
+    const unsigned grid = (unsigned)(n_bg * a.ctas_per_bg);
+    prep_pieces<0><<<grid, kPrepThreads, smem, st>>>(a);
+    prep_scan_local<<<n_bg, kPrepThreads, 0, st>>>(a);
+    prep_scan_global<<<n_bg, kPrepThreads, 0, st>>>(a);
+    prep_pieces<1><<<grid, kPrepThreads, smem, st>>>(a);
+    prep_tile_bounds<<<(unsigned)((a.max_tiles + 7) / 8), 256, 0, st>>>(a);
+    if (launches) *launches += 5;
+    return cudaGetLastError();
+}
+
+}  // namespace tc
+}  // namespace sla

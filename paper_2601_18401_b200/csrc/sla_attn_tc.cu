@@ -13,9 +13,7 @@
 // comparison sort of the queries.  A tile is 128 pieces of one group: their Q rows are gathered into
 // shared memory and the tile walks the key blocks they cover from left to right.
 //
-//   tc_pieces<count>     per row: spans -> pieces, histogram of (group, blocks covered)
-//   tc_scan              prefix sums, tile table
-//   tc_pieces<scatter>   per row: piece records to their sorted places
+//   tc::prepare          the counting sort and the tile table (sla_attn_prep.cu)
 //   tc_attend            persistent CTAs, tiles handed out through an atomic counter; per tile and
 //                        key block: S = Q K^T (tcgen05, smem x smem -> TMEM), row softmax in
 //                        registers, P (bf16) back into TMEM, O += P V (tcgen05, TMEM x smem -> TMEM)
@@ -34,7 +32,7 @@
 #include <stdio.h>
 #endif
 
-#include "sla_kernels.h"
+#include "sla_attn_tc.cuh"
 #include "sla_tc_ptx.cuh"
 
 namespace sla {
@@ -44,8 +42,8 @@ namespace {
 using bf16 = __nv_bfloat16;
 
 constexpr int kD = 128;
-constexpr int kBK = 64;          // keys per block
-constexpr int kRows = 128;       // pieces per tile
+using tc::kBK;    // keys per block
+using tc::kRows;  // pieces per tile
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;
 constexpr uint32_t kColS = 0;    // S buffers at columns 0 and 64
@@ -81,170 +79,12 @@ struct TcParams {
     const int4 *recs;          // sorted piece records {row, j, lo, hi}
     const int4 *tiles;         // {b*Hkv+g, end block, first record, record count | key blocks to walk << 8}
     const int *n_tiles;
-    int *tile_counter;
     __half *part_o;            // [rows*top_k][128] normalised piece outputs, fp16 with one power-of-two
                                // scale per 32-column chunk (block floating point)
     float2 *part_lse;          // [rows*top_k] {log2-domain log-sum-exp of the piece, four chunk exponents}
     int *status;
     int Hkv;
 };
-
-// ------------------------------------------------------------------------------------------------
-// Pieces of one row: spans of the selected anchors (Algorithm 1), sorted by (lo, hi), clipped so
-// that each key is kept once.  Returns the number of pieces; lo[]/hi[] hold them left to right.
-__device__ inline int row_pieces(const int32_t *__restrict__ an, int top_k, long long i, long long ell,
-                                 int back, int fwd, int *lo, int *hi, int *status) {
-    int n = 0;
-    for (int j = 0; j < top_k; ++j) {
-        const long long t = an[j];
-        if (t > i) { atomicOr(status, kStatusBadIndex); continue; }
-        if (t < 0) continue;
-        const long long a = t - (long long)back * ell, z = t + (long long)fwd * ell;
-        const int l0 = (int)(a > 0 ? a : 0), h0 = (int)(z < i ? z : i);
-        int pos = n;   // insertion sort by (lo, hi)
-        while (pos > 0 && (lo[pos - 1] > l0 || (lo[pos - 1] == l0 && hi[pos - 1] > h0))) {
-            lo[pos] = lo[pos - 1];
-            hi[pos] = hi[pos - 1];
-            --pos;
-        }
-        lo[pos] = l0;
-        hi[pos] = h0;
-        ++n;
-    }
-    int cnt = 0;
-    long long next_free = 0;
-    for (int a = 0; a < n; ++a) {
-        const int l0 = lo[a], h0 = hi[a];
-        const long long j0 = l0 > next_free ? l0 : next_free;
-        if (j0 <= h0) {
-            lo[cnt] = (int)j0;
-            hi[cnt] = h0;
-            ++cnt;
-        }
-        if ((long long)h0 + 1 > next_free) next_free = (long long)h0 + 1;
-    }
-    return cnt;
-}
-
-struct PrepParams {
-    const int32_t *anchor;  // [B,Hq,Lq,top_k]
-    int B, Hq, Hkv, G, top_k, span_len, back, fwd;
-    long long Lq, q_pos0, r0;
-    int Lc;                 // query rows of this chunk (per head)
-    int NB, nb_max;         // key blocks, largest number of blocks a piece may cover
-    int *key_count;         // [n_keys] histogram, later the exclusive offsets
-    int *key_cursor;        // [n_keys]
-    int4 *recs;
-    unsigned char *n_pieces;  // [rows]
-    int *status;
-};
-
-// One thread per (b, h, r) row of the chunk.  kScatter = false: count; true: write the records.
-template <bool kScatter>
-__global__ void __launch_bounds__(128) tc_pieces(PrepParams p) {
-    const long long row = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long rows = (long long)p.B * p.Hq * p.Lc;
-    if (row >= rows) return;
-    const int rc = (int)(row % p.Lc);
-    const int bh = (int)(row / p.Lc);
-    const int h = bh % p.Hq, b = bh / p.Hq, g = h / p.G;
-    const long long r = p.r0 + rc;
-    const long long i = p.q_pos0 + r;
-    int lo[kMaxTopK], hi[kMaxTopK];
-    const int32_t *an = p.anchor + (((long long)b * p.Hq + h) * p.Lq + r) * p.top_k;
-    const int cnt = row_pieces(an, p.top_k, i, base_len(i, p.span_len), p.back, p.fwd, lo, hi, p.status);
-    if (!kScatter) p.n_pieces[row] = (unsigned char)cnt;
-    const long long group0 = ((long long)b * p.Hkv + g) * p.NB;
-    for (int j = 0; j < cnt; ++j) {
-        const int eb = hi[j] / kBK, sb = lo[j] / kBK;
-        const long long key = (group0 + eb) * p.nb_max + (eb - sb);
-        if (!kScatter) {
-            atomicAdd(p.key_count + key, 1);
-        } else {
-            const int pos = p.key_count[key] + atomicAdd(p.key_cursor + key, 1);
-            p.recs[pos] = make_int4((int)row, j, lo[j], hi[j]);
-        }
-    }
-}
-
-// Single block: exclusive prefix sum of the key histogram (in place), tiles per group, tile table.
-__global__ void __launch_bounds__(1024)
-tc_scan(int *key_count, long long n_keys, int nb_max, int n_groups, int NB, int4 *tiles, int *n_tiles,
-        int *tile_counter, int max_tiles) {
-    __shared__ int warp_sum[32];
-    __shared__ int carry_s;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    auto block_excl_scan = [&](int v, int &total) -> int {
-        int x = v;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int y = __shfl_up_sync(0xffffffffu, x, off);
-            if (lane >= off) x += y;
-        }
-        if (lane == 31) warp_sum[warp] = x;
-        __syncthreads();
-        if (warp == 0) {
-            int w = warp_sum[lane];
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int y = __shfl_up_sync(0xffffffffu, w, off);
-                if (lane >= off) w += y;
-            }
-            warp_sum[lane] = w;
-        }
-        __syncthreads();
-        total = warp_sum[31];
-        const int base = warp > 0 ? warp_sum[warp - 1] : 0;
-        __syncthreads();
-        return base + x - v;
-    };
-    // pass 1: key offsets
-    const long long per = (n_keys + 1023) / 1024;
-    const long long k0 = per * tid, k1 = (k0 + per < n_keys) ? k0 + per : n_keys;
-    int local = 0;
-    for (long long k = k0; k < k1; ++k) local += key_count[k];
-    int total;
-    int run = block_excl_scan(local, total);
-    for (long long k = k0; k < k1; ++k) {
-        const int c = key_count[k];
-        key_count[k] = run;
-        run += c;
-    }
-    __syncthreads();
-    const int n_recs = total;
-    // pass 2: tiles per group (a group's records are contiguous: keys group*nb_max .. +nb_max-1)
-    if (tid == 0) carry_s = 0;
-    __syncthreads();
-    for (int g0 = 0; g0 < n_groups; g0 += 1024) {
-        const int g = g0 + tid;
-        int first = 0, cnt = 0;
-        if (g < n_groups) {
-            first = key_count[(long long)g * nb_max];
-            const int last = (g + 1 < n_groups) ? key_count[(long long)(g + 1) * nb_max] : n_recs;
-            cnt = last - first;
-        }
-        const int nt = (cnt + kRows - 1) / kRows;
-        int tot;
-        const int off = block_excl_scan(nt, tot) + carry_s;
-        int cls = 0;   // class (blocks covered - 1) of the record the walk below has reached
-        for (int t = 0; t < nt; ++t) {
-            const int idx = off + t;
-            const int left = cnt - t * kRows;
-            const int n_here = left < kRows ? left : kRows;
-            // records of a group are ordered by blocks covered, so the tile's last record covers most
-            const int last = first + t * kRows + n_here - 1;
-            while (cls + 1 < nb_max && key_count[(long long)g * nb_max + cls + 1] <= last) ++cls;
-            if (idx < max_tiles) tiles[idx] = make_int4(g / NB, g % NB, first + t * kRows, n_here | ((cls + 1) << 8));
-        }
-        __syncthreads();
-        if (tid == 0) carry_s += tot;
-        __syncthreads();
-    }
-    if (tid == 0) {
-        *n_tiles = carry_s < max_tiles ? carry_s : max_tiles;
-        *tile_counter = 0;
-    }
-}
 
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -762,20 +602,26 @@ bool tc_attention_supported(const Call &c, int dtype) {
 TcPlan plan_attention_tc(const Call &c, int Lc) {
     TcPlan p;
     p.Lc = Lc;
+    p.n_bg = c.B * c.Hkv;
     p.NB = (int)((c.Lkv + kBK - 1) / kBK);
     const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     if (span_tokens > c.Lkv) span_tokens = c.Lkv;
     p.nb_max = (int)((span_tokens - 1) / kBK + 2);
-    p.n_groups = (long long)c.B * c.Hkv * p.NB;
-    p.n_keys = p.n_groups * p.nb_max;
+    // pieces of a group are ordered by blocks covered, in as many classes as the CTA-local histogram
+    // of the counting sort affords (NB * ncls counters in shared memory)
+    p.ncls = p.nb_max < 8 ? p.nb_max : 8;
+    while (p.ncls > 1 && (size_t)p.NB * p.ncls * 4 > 160 * 1024) p.ncls /= 2;
+    p.ok = (size_t)p.NB * p.ncls * 4 <= 160 * 1024;
+    p.ctas_per_bg = (148 + p.n_bg - 1) / p.n_bg;
     const size_t rows = (size_t)c.B * c.Hq * Lc;
     const size_t slots = rows * c.top_k;
-    p.max_tiles = (long long)(slots / kRows) + p.n_groups + 1;
+    const size_t n_keys = (size_t)p.n_bg * p.NB * p.ncls;
+    p.max_tiles = (long long)(slots / kRows) + (long long)p.n_bg * p.NB + 1;
     size_t off = 0;
-    p.off_counters = off; off = align256(off + 64);
-    p.off_key_count = off; off = align256(off + (size_t)p.n_keys * 4);
-    p.off_key_cursor = off; off = align256(off + (size_t)p.n_keys * 4);
+    p.off_counters = off; off = align256(off + 64 + (size_t)p.n_bg * 8);
+    p.off_key_count = off; off = align256(off + n_keys * 4);
+    p.off_key_cursor = off; off = align256(off + n_keys * 4);
     p.off_tiles = off; off = align256(off + (size_t)p.max_tiles * 16);
     p.off_recs = off; off = align256(off + slots * 16);
     p.off_npieces = off; off = align256(off + rows);
@@ -795,8 +641,8 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         Lc = (Lc + 1) / 2;
         plan = plan_attention_tc(c, (int)Lc);
     }
-    if (plan.bytes > scratch_bytes) return cudaErrorMemoryAllocation;
-    if (plan.n_keys > (1ll << 30) || (long long)c.B * c.Hq * Lc * c.top_k > (1ll << 31) - 1) return cudaErrorInvalidValue;
+    if (plan.bytes > scratch_bytes || !plan.ok) return cudaErrorMemoryAllocation;
+    if (plan.max_tiles > (1ll << 30) || (long long)c.B * c.Hq * Lc * c.top_k > (1ll << 31) - 1) return cudaErrorInvalidValue;
 
     CUtensorMap tm_k, tm_v;
     int slot[3];
@@ -814,35 +660,37 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         const long long rows = (long long)c.B * c.Hq * lc;
         cudaError_t e = cudaMemsetAsync(ws + plan.off_key_count, 0, plan.off_tiles - plan.off_key_count, st);
         if (e != cudaSuccess) return e;
-        PrepParams pp;
-        pp.anchor = anchor; pp.B = c.B; pp.Hq = c.Hq; pp.Hkv = c.Hkv; pp.G = c.G; pp.top_k = c.top_k;
-        pp.span_len = c.span_len; pp.back = c.back; pp.fwd = c.fwd; pp.Lq = c.Lq; pp.q_pos0 = c.q_pos0;
-        pp.r0 = r0; pp.Lc = lc; pp.NB = plan.NB; pp.nb_max = plan.nb_max;
-        pp.key_count = (int *)(ws + plan.off_key_count);
-        pp.key_cursor = (int *)(ws + plan.off_key_cursor);
-        pp.recs = (int4 *)(ws + plan.off_recs);
-        pp.n_pieces = (unsigned char *)(ws + plan.off_npieces);
-        pp.status = c.status;
-        const unsigned blocks = (unsigned)((rows + 127) / 128);
-        tc_pieces<false><<<blocks, 128, 0, st>>>(pp);
-        tc_scan<<<1, 1024, 0, st>>>(pp.key_count, plan.n_keys, plan.nb_max, (int)plan.n_groups, plan.NB,
-                                    (int4 *)(ws + plan.off_tiles), counters, counters + 1, (int)plan.max_tiles);
-        tc_pieces<true><<<blocks, 128, 0, st>>>(pp);
+        tc::PrepArgs pa;
+        pa.anchor = anchor; pa.B = c.B; pa.Hq = c.Hq; pa.Hkv = c.Hkv; pa.G = c.G; pa.top_k = c.top_k;
+        pa.span_len = c.span_len; pa.back = c.back; pa.fwd = c.fwd; pa.Lq = c.Lq; pa.q_pos0 = c.q_pos0;
+        pa.r0 = r0; pa.Lc = lc; pa.NB = plan.NB; pa.nb_max = plan.nb_max; pa.ncls = plan.ncls;
+        pa.ctas_per_bg = plan.ctas_per_bg;
+        pa.key_count = (int *)(ws + plan.off_key_count);
+        pa.key_cursor = (int *)(ws + plan.off_key_cursor);
+        pa.totals = counters + 16;
+        pa.n_tiles = counters;
+        pa.tiles = (int4 *)(ws + plan.off_tiles);
+        pa.max_tiles = (int)plan.max_tiles;
+        pa.recs = (int4 *)(ws + plan.off_recs);
+        pa.n_pieces = (unsigned char *)(ws + plan.off_npieces);
+        pa.status = c.status;
+        e = tc::prepare(pa, st, launches);
+        if (e != cudaSuccess) return e;
         TcParams tp;
         tp.q = (const bf16 *)q; tp.q_sb = c.q_sb; tp.q_sh = c.q_sh; tp.q_st = c.q_st;
         tp.Hq = c.Hq; tp.G = c.G; tp.Lc = lc; tp.top_k = c.top_k; tp.r0 = r0;
         tp.scale2 = c.softmax_scale * kLog2e;
         tp.slot_t = slot[0]; tp.slot_h = slot[1]; tp.slot_b = slot[2];
-        tp.recs = pp.recs; tp.tiles = (const int4 *)(ws + plan.off_tiles);
-        tp.n_tiles = counters; tp.tile_counter = counters + 1;
+        tp.recs = pa.recs; tp.tiles = pa.tiles;
+        tp.n_tiles = counters;
         tp.part_o = (__half *)(ws + plan.off_part_o); tp.part_lse = (float2 *)(ws + plan.off_part_lse);
         tp.status = c.status; tp.Hkv = c.Hkv;
         tc_attend<<<2 * sm_count, kThreads, kSmemBytes, st>>>(tm_k, tm_v, tp);
         const unsigned mblocks = (unsigned)((rows * 16 + 255) / 256);
-        tc_merge<<<mblocks, 256, 0, st>>>(tp.part_o, tp.part_lse, pp.n_pieces, c, lc, r0, (bf16 *)out, lse);
+        tc_merge<<<mblocks, 256, 0, st>>>(tp.part_o, tp.part_lse, pa.n_pieces, c, lc, r0, (bf16 *)out, lse);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
-        if (launches) *launches += 5;
+        if (launches) *launches += 2;
     }
     return cudaSuccess;
 }

@@ -19,8 +19,9 @@ cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int
 // ---- tensor-core span-attention for prefill, bf16 / head_dim 128 (sla_attn_tc.cu) ---------------
 // Scratch layout for one chunk of Lc query positions (all offsets in bytes).
 struct TcPlan {
-    int Lc, NB, nb_max;
-    long long n_groups, n_keys, max_tiles;
+    int Lc, n_bg, NB, nb_max, ncls, ctas_per_bg;
+    bool ok;   // false when the shared-memory histogram of the counting sort cannot hold NB buckets
+    long long max_tiles;
     size_t off_counters, off_key_count, off_key_cursor, off_tiles, off_recs, off_npieces, off_part_lse,
         off_part_o, bytes;
 };
