@@ -36,6 +36,9 @@ from paper_2601_18401_b200 import synth
 
 METRIC = "prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one tc_attend launch, from the ncu capture summarised
+# in profiles/ (taken on a quarter-length case and scaled by the number of tiles); None until measured
+TC_ATTEND_DRAM_BYTES_PER_LAUNCH = None
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -53,48 +56,53 @@ def load_peaks():
 
 # ------------------------------------------------------------------------------------ clocks
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons in the background during the timed region."""
+    """Samples SM clock and throttle reasons through NVML (read-only) in a background thread during
+    the timed region; falls back to one nvidia-smi query when NVML is not importable."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
+        self.index, self.samples, self.masks, self.max_mhz = index, [], [], None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                self.masks.append(int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)))
+            except Exception:
+                pass
+            time.sleep(0.004)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            threading.Thread(target=self._pump, daemon=True).start()
-        except OSError:
-            self.proc = None
-
-    def _pump(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            parts = [x.strip() for x in ln.split(",")]
-            if len(parts) < 6:
-                continue
+        if self.nv is None:
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[2:6]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        busy = sorted(sm)[len(sm) // 2:] if sm else []   # upper half: samples taken under load
-        return {"sm_mhz": float(np.median(busy)) if busy else None,
-                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+                out = subprocess.run(["nvidia-smi", f"--id={self.index}", "--query-gpu=clocks.sm,clocks.max.sm",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True).stdout
+                a, b = [float(x) for x in out.strip().split(",")]
+                return {"sm_mhz": a, "sm_max_mhz": b, "reasons": ["nvml unavailable: one nvidia-smi sample after the run"]}
+            except Exception:
+                return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source"]}
+        self._stop.set()
+        self._thread.join(timeout=1.0)
+        reasons = sorted({name for m in self.masks for bit, name in self.REASONS.items() if m & bit})
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(self.samples)}
 
 
 # ------------------------------------------------------------------------------------ bookkeeping
@@ -258,6 +266,7 @@ def run_ours(args, w):
     for _ in range(max(3, args.warmup)):
         step()
     torch.cuda.synchronize()
+    sla.sla_set_kernel_timing(handle, True)   # events around the main attention kernel, on its stream
     launches0 = sla.sla_kernel_launches(handle)
     sampler = ClockSampler(local)
     sampler.start()
@@ -277,6 +286,9 @@ def run_ours(args, w):
     launches = sla.sla_kernel_launches(handle) - launches0
     total_ms = t0.elapsed_time(t1)
     attn_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    kern_ms_sum, kern_n = sla.sla_kernel_time_ms(handle)
+    sla.sla_set_kernel_timing(handle, False)
+    kern_ms = kern_ms_sum / args.steps if kern_n else attn_ms   # generic path: whole call
     if dist:
         t = torch.tensor([total_ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -287,12 +299,16 @@ def run_ours(args, w):
     # roofline of the dominant kernel (span-attention): 4*D flops per attended (query, key) pair
     pairs = attended_pairs(anchor, w.span_len, w.back_factor, w.fwd_factor)
     flops = 4.0 * D * pairs
-    tflops = flops / (attn_ms * 1e-3) / 1e12
+    tflops = flops / (kern_ms * 1e-3) / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
-    roofline = {"bound": "tensor", "kernel": "sla_span_attention", "achieved": tflops, "peak": peak_tf,
-                "unit": "TFLOP/s", "frac": tflops / peak_tf, "traffic": None, "flops_per_launch": flops,
-                "ms_per_launch": attn_ms, "search_ms_per_launch": ms_per_step - attn_ms,
-                "peak_source": peaks["_source"] + " (sustained bf16 matmul)"}
+    roofline = {"bound": "tensor", "kernel": "tc_attend (tcgen05 span-attention)" if kern_n else "attn_rows_simt",
+                "achieved": tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": tflops / peak_tf,
+                "traffic": TC_ATTEND_DRAM_BYTES_PER_LAUNCH if kern_n else None,
+                "flops_per_launch": flops, "ms_per_launch": kern_ms, "launches_timed": kern_n,
+                "whole_call": {"sla_span_attention_ms": attn_ms, "sla_span_search_ms": ms_per_step - attn_ms,
+                               "attention_tflops": flops / (attn_ms * 1e-3) / 1e12,
+                               "attention_frac": flops / (attn_ms * 1e-3) / 1e12 / peak_tf},
+                "peak_source": peaks["_source"] + " (sustained bf16 matmul; the kernel runs inside a long step)"}
 
     # end to end through the host-buffer C call: pinned host inputs, host outputs, copies inside
     host = {n: t.cpu().pin_memory() for n, t in x.items()}
@@ -355,11 +371,11 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, help="index into the benchmark configurations (prefill ones)")
-    ap.add_argument("--ref-rows", type=int, default=1024, help="query positions the CPU oracle is timed on")
+    ap.add_argument("--ref-rows", type=int, default=4096, help="query positions the CPU oracle is timed on")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="short decode loops (for smoke runs)")

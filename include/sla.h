@@ -123,6 +123,14 @@ sla_status_t sla_poll_status(sla_handle_t handle, void *stream);
  * paper has no counterpart).  Host-only. */
 int64_t sla_kernel_launches(sla_handle_t handle);
 
+/* Device-side timing of the dominant kernel (a diagnostic for benchmarks; the paper has no
+ * counterpart).  With timing enabled, sla_span_attention brackets its main attention kernel with
+ * CUDA events on the caller's stream (at most 64 launches are kept between two reads);
+ * sla_kernel_time_ms waits for them, returns the summed milliseconds of the launches recorded since
+ * the previous read and how many they were (n_launches may be NULL), and starts over. */
+sla_status_t sla_set_kernel_timing(sla_handle_t handle, int enable);
+sla_status_t sla_kernel_time_ms(sla_handle_t handle, float *ms, int32_t *n_launches);
+
 /* ---- span-search (Section "Span search"; Algorithm 1 scoring and TopK lines) -------------- */
 
 /* Query row r (0 <= r < Lq) is position i = q_pos0 + r; keys 0 .. Lkv-1 are valid; requires

@@ -23,7 +23,8 @@ SLA_UNION, SLA_PER_SPAN = 0, 1
 EXPORTS = [
     "sla_create", "sla_destroy", "sla_workspace_bytes", "sla_status_string", "sla_last_error",
     "sla_poll_status", "sla_span_search", "sla_span_attention", "sla_decode_step",
-    "sla_host_staging_bytes", "sla_prefill_host", "sla_kernel_launches",
+    "sla_host_staging_bytes", "sla_prefill_host", "sla_kernel_launches", "sla_set_kernel_timing",
+    "sla_kernel_time_ms",
 ]
 
 
@@ -81,6 +82,10 @@ def load_library():
     lib.sla_decode_step.argtypes = [vp, vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
     lib.sla_kernel_launches.restype = i64
     lib.sla_kernel_launches.argtypes = [vp]
+    lib.sla_set_kernel_timing.restype = i32
+    lib.sla_set_kernel_timing.argtypes = [vp, i32]
+    lib.sla_kernel_time_ms.restype = i32
+    lib.sla_kernel_time_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.sla_host_staging_bytes.restype = sz
     lib.sla_host_staging_bytes.argtypes = [LP, PP, i64]
     lib.sla_prefill_host.restype = i32
@@ -166,6 +171,17 @@ def sla_host_staging_bytes(layout: sla_layout_t, params: sla_params_t, L: int) -
 
 def sla_kernel_launches(handle: Handle) -> int:
     return int(handle._lib.sla_kernel_launches(handle.ptr))
+
+
+def sla_set_kernel_timing(handle: Handle, enable: bool) -> None:
+    handle.check(handle._lib.sla_set_kernel_timing(handle.ptr, int(bool(enable))), "sla_set_kernel_timing")
+
+
+def sla_kernel_time_ms(handle: Handle):
+    """(milliseconds, launches) of the main attention kernel since the previous read."""
+    ms, n = C.c_float(0.0), C.c_int32(0)
+    handle.check(handle._lib.sla_kernel_time_ms(handle.ptr, C.byref(ms), C.byref(n)), "sla_kernel_time_ms")
+    return float(ms.value), int(n.value)
 
 
 def sla_poll_status(handle: Handle, stream=None) -> int:

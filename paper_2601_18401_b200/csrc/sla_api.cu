@@ -15,6 +15,7 @@ struct sla_handle_s {
     size_t ws_bytes = 0;
     long long launches = 0;   // kernels launched through this handle
     size_t scratch_avail = 0; // bytes of workspace after the header that kernels may use as scratch
+    sla::KernelTimer timer;   // sla_set_kernel_timing / sla_kernel_time_ms
     bool force_simt = false;  // environment SLA_FORCE_SIMT=1: generic kernels only (for A/B checks)
     char err[256] = {0};
 };
@@ -108,6 +109,32 @@ const char *sla_last_error(sla_handle_t h) { return h ? h->err : "NULL handle"; 
 
 int64_t sla_kernel_launches(sla_handle_t h) { return h ? h->launches : 0; }
 
+sla_status_t sla_set_kernel_timing(sla_handle_t h, int enable) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (enable && !h->timer.ev[0]) {
+        for (int j = 0; j < 2 * sla::KernelTimer::kMaxPairs; ++j)
+            if (cudaEventCreate(&h->timer.ev[j]) != cudaSuccess) return cuda_fail(h, cudaGetLastError(), "sla_set_kernel_timing");
+    }
+    h->timer.enabled = enable != 0;
+    h->timer.used = 0;
+    return SLA_OK;
+}
+
+sla_status_t sla_kernel_time_ms(sla_handle_t h, float *ms, int32_t *n_launches) {
+    if (!h || !ms) return SLA_ERR_INVALID_ARG;
+    *ms = 0.f;
+    if (n_launches) *n_launches = h->timer.used;
+    for (int j = 0; j < h->timer.used; ++j) {
+        float t = 0.f;
+        cudaError_t e = cudaEventSynchronize(h->timer.ev[2 * j + 1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t, h->timer.ev[2 * j], h->timer.ev[2 * j + 1]);
+        if (e != cudaSuccess) return cuda_fail(h, e, "sla_kernel_time_ms");
+        *ms += t;
+    }
+    h->timer.used = 0;
+    return SLA_OK;
+}
+
 sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes) {
     if (!handle) return SLA_ERR_INVALID_ARG;
     *handle = nullptr;
@@ -139,6 +166,8 @@ sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes
 
 sla_status_t sla_destroy(sla_handle_t h) {
     if (!h) return SLA_ERR_INVALID_ARG;
+    for (int j = 0; j < 2 * sla::KernelTimer::kMaxPairs; ++j)
+        if (h->timer.ev[j]) cudaEventDestroy(h->timer.ev[j]);
     cudaError_t e = cudaFree(h->ws);
     delete h;
     return e == cudaSuccess ? SLA_OK : SLA_ERR_CUDA;
@@ -211,7 +240,7 @@ sla_status_t sla_span_attention(sla_handle_t h, const void *q, const void *k, co
         const sla::TcPlan probe = sla::plan_attention_tc(c, (int)min_chunk);
         if (probe.ok && probe.bytes <= h->scratch_avail) {
             cudaError_t e = sla::launch_attn_tc(q, k, v, c, anchor, out, lse, h->ws + kHeaderBytes,
-                                                h->scratch_avail, h->sm_count, st, &h->launches);
+                                                h->scratch_avail, h->sm_count, st, &h->launches, &h->timer);
             if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_attention (tensor-core path)");
             return SLA_OK;
         }

@@ -633,7 +633,7 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
 
 cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor,
                            void *out, float *lse, void *scratch, size_t scratch_bytes, int sm_count,
-                           cudaStream_t st, long long *launches) {
+                           cudaStream_t st, long long *launches, KernelTimer *timer) {
     // the largest chunk of query positions whose scratch fits
     long long Lc = c.Lq;
     TcPlan plan = plan_attention_tc(c, (int)Lc);
@@ -685,7 +685,9 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         tp.n_tiles = counters;
         tp.part_o = (__half *)(ws + plan.off_part_o); tp.part_lse = (float2 *)(ws + plan.off_part_lse);
         tp.status = c.status; tp.Hkv = c.Hkv;
+        if (timer) timer->begin(st);
         tc_attend<<<2 * sm_count, kThreads, kSmemBytes, st>>>(tm_k, tm_v, tp);
+        if (timer) timer->end(st);
         const unsigned mblocks = (unsigned)((rows * 16 + 255) / 256);
         tc_merge<<<mblocks, 256, 0, st>>>(tp.part_o, tp.part_lse, pa.n_pieces, c, lc, r0, (bf16 *)out, lse);
         e = cudaGetLastError();

@@ -11,6 +11,16 @@ cudaError_t launch_search_simt(const void *q_s, const void *k, const Call &c, in
 cudaError_t launch_attn_simt(const void *q, const void *k, const void *v, const Call &c, int dtype,
                              const int32_t *anchor, void *out, float *lse, cudaStream_t st);
 
+// Optional device-side timing of the dominant kernel of a call (CUDA events on the caller's stream).
+struct KernelTimer {
+    static constexpr int kMaxPairs = 64;
+    bool enabled = false;
+    int used = 0;                       // event pairs recorded by the last call
+    cudaEvent_t ev[2 * kMaxPairs] = {};
+    void begin(cudaStream_t st) { if (enabled && used < kMaxPairs) cudaEventRecord(ev[2 * used], st); }
+    void end(cudaStream_t st) { if (enabled && used < kMaxPairs) { cudaEventRecord(ev[2 * used + 1], st); ++used; } }
+};
+
 // ---- tensor-core span-search for bf16 / head_dim 128 (sla_search_mma.cu) -------------------------
 bool search_mma_supported(const Call &c, int dtype);
 cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int32_t *out_anchor, float *out_score,
@@ -32,7 +42,7 @@ TcPlan plan_attention_tc(const Call &c, int Lc);
 // *launches.  Returns cudaErrorMemoryAllocation when not even one query position fits.
 cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor,
                            void *out, float *lse, void *scratch, size_t scratch_bytes, int sm_count,
-                           cudaStream_t st, long long *launches);
+                           cudaStream_t st, long long *launches, KernelTimer *timer);
 
 // ---- decode step (sla_decode.cu) ---------------------------------------------------------------
 // Scratch layout of one decode step, all offsets in bytes from the scratch base.
