@@ -18,10 +18,11 @@ def code_of(t: torch.Tensor) -> int:
 def compare_search(anchor_gpu, score_gpu, ref, q_pos0=0, rows=None):
     """Selected anchors must equal the oracle's as sets on every clear-cut row; returns the number of
     exempt near-tie rows.  On every row the GPU's anchors must be valid candidates."""
+    if rows is not None:   # slice on the device: the full tensors can be gigabytes
+        idx = torch.as_tensor(np.asarray(rows), device=anchor_gpu.device)
+        anchor_gpu, score_gpu = anchor_gpu[:, :, idx], score_gpu[:, :, idx]
     a = anchor_gpu.cpu().numpy()
     s = score_gpu.cpu().numpy().astype(np.float64)
-    if rows is not None:
-        a, s = a[:, :, rows], s[:, :, rows]
     ra, rs, gap = ref["anchor"], ref["score"], ref["gap"]
     assert a.shape == ra.shape
     clear = gap > TIE_GAP
@@ -48,19 +49,20 @@ def compare_search(anchor_gpu, score_gpu, ref, q_pos0=0, rows=None):
 
 
 def oracle_attention_for(x_host, dtype_code, anchor_gpu, w, q_pos0=0, rows=None, softmax_scale=None):
-    a = anchor_gpu.cpu().numpy()
     if rows is not None:
-        a = np.ascontiguousarray(a[:, :, rows])
+        anchor_gpu = anchor_gpu[:, :, torch.as_tensor(np.asarray(rows), device=anchor_gpu.device)]
+    a = np.ascontiguousarray(anchor_gpu.cpu().numpy())
     return O.span_attention(x_host["q"], x_host["k"], x_host["v"], dtype_code, a, span_len=w.span_len,
                             back_factor=w.back_factor, fwd_factor=w.fwd_factor, q_pos0=q_pos0, rows=rows,
                             softmax_scale=softmax_scale)
 
 
 def compare_attention(out_gpu, lse_gpu, ref, dtype_name, rows=None):
+    if rows is not None:
+        idx = torch.as_tensor(np.asarray(rows), device=out_gpu.device)
+        out_gpu, lse_gpu = out_gpu[:, :, idx], lse_gpu[:, :, idx]
     o = out_gpu.float().cpu().numpy().astype(np.float64)
     l = lse_gpu.cpu().numpy().astype(np.float64)
-    if rows is not None:
-        o, l = o[:, :, rows], l[:, :, rows]
     tol = OUT_TOL[dtype_name]
     err = np.abs(o - ref["out"]).max()
     assert err <= tol, f"output max-abs error {err} above {tol}"

@@ -1,0 +1,159 @@
+"""GPU parity at the full sizes of the benchmark configurations, in the launch configuration the
+benchmark times (whole sequence per call, workspace from sla_workspace_bytes), checked on sampled
+rows the oracle computes one by one, plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import parity_util as P
+from oracle import sla_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sla():
+    import paper_2601_18401_b200 as sla_pkg
+    return sla_pkg
+
+
+def sample_rows(L, seed, n_random=192):
+    """Stratified sample: the first and last rows, tile edges, and seeded random positions."""
+    rng = np.random.default_rng(seed)
+    rows = set(range(0, 48)) | set(range(L - 48, L))
+    rows |= {int(x) for x in rng.integers(0, L, n_random)}
+    rows |= {int(x) for x in rng.integers(0, L // 128, 24) * 128} | {int(x) for x in rng.integers(1, L // 128, 24) * 128 - 1}
+    return np.array(sorted(rows), dtype=np.int64)
+
+
+def run_prefill_config(sla, w, seed):
+    from paper_2601_18401_b200 import synth
+    dev = "cuda:0"
+    x = synth.make_prefill(w, device=dev)
+    params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim)
+    layout = sla.make_layout(x["q"], x["k"])
+    handle = sla.Handle(0, sla.sla_workspace_bytes(layout, params, w.seq_len, w.seq_len) + (64 << 20))
+    anchor, score = sla.sla_span_search(handle, x["q_s"], x["k"], params)
+    out, lse = sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    # properties at full size: anchors are valid stride positions, scores sorted, padding consistent
+    a64 = anchor.to(torch.int64)
+    i = torch.arange(w.seq_len, device=dev)[None, None, :, None]
+    d = i + 1 - a64
+    m = torch.sqrt(d.clamp(min=0).double()).round().to(torch.int64)
+    assert bool(torch.all((a64 == -1) | ((m * m == d) & (m >= 1) & (a64 >= 0))))
+    assert bool(torch.all(score[..., :-1] >= score[..., 1:]))
+    n_anchor = torch.sqrt((i + 1).double()).floor().to(torch.int64)
+    assert bool(torch.all((a64 >= 0).sum(-1, keepdim=True) == n_anchor.clamp(max=w.top_k)))
+    assert bool(torch.isfinite(out.float()).all()) and bool(torch.isfinite(lse).all())
+    # sampled rows against the oracle
+    rows = sample_rows(w.seq_len, seed)
+    host = P.host_inputs(x)
+    code = synth.dtype_code(w.dtype)
+    ref_s = O.span_search(host["q_s"], host["k"], code, top_k=w.top_k, rows=rows)
+    ties = P.compare_search(anchor, score, ref_s, rows=rows)
+    ref_a = P.oracle_attention_for(host, code, anchor, w, rows=rows)
+    err, lerr = P.compare_attention(out, lse, ref_a, w.dtype, rows=rows)
+    handle.close()
+    return dict(ties=ties, rows=len(rows), err=err, lerr=lerr)
+
+
+def test_prefill_L65536_planted(sla):
+    """Second benchmark configuration: 32/8 heads, L = 65536, bf16, 16 planted spans, l = 256, k = 8."""
+    from paper_2601_18401_b200 import synth
+    r = run_prefill_config(sla, synth.CONFIGS[1], seed=11)
+    print("prefill_L65536:", r)
+    assert r["ties"] <= 0.02 * r["rows"] * 32
+
+
+def test_prefill_stress_L262144(sla):
+    """Third benchmark configuration: batch 2, 16/4 heads, L = 262144, l = 512, k = 16."""
+    from paper_2601_18401_b200 import synth
+    r = run_prefill_config(sla, synth.CONFIGS[2], seed=12)
+    print("prefill_stress:", r)
+    assert r["ties"] <= 0.05 * r["rows"] * 32
+
+
+def _decode_check(sla, handle, w, kc, vc, hk, hv, n_ctx, step_inputs, sparse_fill=None):
+    from paper_2601_18401_b200 import synth
+    params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
+    out, lse, anchor, score = sla.sla_decode_step(handle, step_inputs["q_s"], step_inputs["q"], kc, vc, n_ctx, params)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    code = synth.dtype_code(w.dtype)
+    q_s = synth.to_numpy(step_inputs["q_s"])[:, :, None]
+    q = synth.to_numpy(step_inputs["q"])[:, :, None]
+    if sparse_fill is not None:
+        sparse_fill(anchor_rows=True)
+    ref_s = O.span_search(q_s, hk, code, top_k=w.top_k, q_pos0=n_ctx - 1, Lkv=n_ctx)
+    P.compare_search(anchor[:, :, None], score[:, :, None], ref_s, q_pos0=n_ctx - 1)
+    if sparse_fill is not None:
+        sparse_fill(anchors=anchor.cpu().numpy())
+    att = O.span_attention(q, hk, hv, code, anchor.cpu().numpy()[:, :, None], span_len=w.span_len,
+                           q_pos0=n_ctx - 1, Lkv=n_ctx)
+    return P.compare_attention(out[:, :, None], lse[:, :, None], att, w.dtype)
+
+
+def test_decode_1M(sla):
+    """Fourth configuration: decode at 1,048,576 tokens of context, 32/4 heads, l = 1024, k = 16."""
+    from paper_2601_18401_b200 import synth
+    w = synth.CONFIGS[3]
+    dev = "cuda:0"
+    steps = 6
+    kc, vc = synth.make_decode_cache(w, dev, capacity=w.seq_len + steps)
+    hk, hv = synth.to_numpy(kc), synth.to_numpy(vc)
+    layout = sla.make_layout(torch.empty(1, 32, 128, dtype=torch.bfloat16, device=dev), kc, decode=True)
+    params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
+    handle = sla.Handle(0, sla.sla_workspace_bytes(layout, params, 1, w.seq_len + steps) + (16 << 20))
+    for s in range(steps):
+        x = synth.make_decode_step_inputs(w, s, dev)
+        n_ctx = w.seq_len + s + 1
+        kc[:, :, n_ctx - 1] = x["k_new"]
+        vc[:, :, n_ctx - 1] = x["v_new"]
+        hk[:, :, n_ctx - 1] = synth.to_numpy(x["k_new"])
+        hv[:, :, n_ctx - 1] = synth.to_numpy(x["v_new"])
+        err, lerr = _decode_check(sla, handle, w, kc, vc, hk, hv, n_ctx, x)
+        assert err <= 1e-2
+    handle.close()
+
+
+def test_decode_10M(sla):
+    """Fifth configuration: decode at 10,485,760 tokens of context (21.5 GB of cache), l = 3072,
+    k = 16.  The host copy for the oracle is sparse: only the rows a step touches are fetched."""
+    from paper_2601_18401_b200 import synth
+    w = synth.CONFIGS[4]
+    dev = "cuda:0"
+    free, _ = torch.cuda.mem_get_info()
+    if free < 30 << 30:
+        pytest.skip("needs 30 GB of free device memory")
+    steps = 2
+    cap = w.seq_len + steps
+    kc, vc = synth.make_decode_cache(w, dev, capacity=cap)
+    shape = (w.batch, w.n_kv_heads, cap, w.head_dim)
+    hk, hv = np.empty(shape, dtype=np.uint16), np.empty(shape, dtype=np.uint16)   # pages are touched lazily
+    layout = sla.make_layout(torch.empty(1, 32, 128, dtype=torch.bfloat16, device=dev), kc, decode=True)
+    params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
+    handle = sla.Handle(0, sla.sla_workspace_bytes(layout, params, 1, cap) + (16 << 20))
+    span = w.back_factor * w.span_len
+    for s in range(steps):
+        x = synth.make_decode_step_inputs(w, s, dev)
+        n_ctx = w.seq_len + s + 1
+        kc[:, :, n_ctx - 1] = x["k_new"]
+        vc[:, :, n_ctx - 1] = x["v_new"]
+
+        def fill(anchor_rows=False, anchors=None, n_ctx=n_ctx):
+            i = n_ctx - 1
+            if anchor_rows:
+                m = np.arange(1, int(np.floor(np.sqrt(i + 1))) + 1, dtype=np.int64)
+                t = torch.from_numpy(i + 1 - m * m).to(dev)
+                hk[:, :, t.cpu().numpy()] = synth.to_numpy(kc[:, :, t])
+            if anchors is not None:
+                for tpos in np.unique(anchors[anchors >= 0]):
+                    lo, hi = max(0, int(tpos) - span), int(tpos)
+                    hk[:, :, lo:hi + 1] = synth.to_numpy(kc[:, :, lo:hi + 1])
+                    hv[:, :, lo:hi + 1] = synth.to_numpy(vc[:, :, lo:hi + 1])
+
+        err, lerr = _decode_check(sla, handle, w, kc, vc, hk, hv, n_ctx, x, sparse_fill=fill)
+        assert err <= 1e-2
+    handle.close()
