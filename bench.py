@@ -225,6 +225,39 @@ def bench_decode(sla, handle, w, steps, peaks, dev):
                          "traffic": None, "peak_source": peaks["_source"]}}
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """The slowest rank's figure (every multi-rank number is a max over ranks); identity without dist."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([float(value)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_workload(w, rank: int):
+    """Every rank works on its own sequence: same shapes, its own seed (weak scaling, no exchange)."""
+    return w.scaled(seed=w.seed + 7919 * rank)
+
+
+def measure_e2e(sla, handle, host, params, args, dist, dev, world, B, L):
+    """The same step through sla_prefill_host: pinned host inputs in, host outputs out, all copies
+    inside the timed region."""
+    ho = sla.sla_prefill_host(handle, host["q_s"], host["q"], host["k"], host["v"], params)
+    n_e2e = max(2, min(args.steps, 5))
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    tt = time.perf_counter()
+    for _ in range(n_e2e):
+        sla.sla_prefill_host(handle, host["q_s"], host["q"], host["k"], host["v"], params,
+                             out=ho[0], lse=ho[1], anchor=ho[2], score=ho[3])
+    e2e_s = max_over_ranks((time.perf_counter() - tt) / n_e2e, dist, dev)
+    h2d = sum(host[n].numel() * host[n].element_size() for n in ("q_s", "q", "k", "v"))
+    d2h = sum(t.numel() * t.element_size() for t in ho)
+    return {"value": world * B * L / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": e2e_s * 1e3}
+
+
 def run_ours(args, w):
     import paper_2601_18401_b200 as sla
     rank = int(os.environ.get("RANK", "0"))
@@ -242,7 +275,7 @@ def run_ours(args, w):
     sla.load_library()
     peaks = load_peaks()
 
-    wr = w.scaled(seed=w.seed + 7919 * rank)      # every rank its own sequence
+    wr = rank_workload(w, rank)
     x = synth.make_prefill(wr, device=dev)
     params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim)
     layout = sla.make_layout(x["q"], x["k"])
@@ -289,10 +322,7 @@ def run_ours(args, w):
     kern_ms_sum, kern_n = sla.sla_kernel_time_ms(handle)
     sla.sla_set_kernel_timing(handle, False)
     kern_ms = kern_ms_sum / args.steps if kern_n else attn_ms   # generic path: whole call
-    if dist:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
     value = world * B * L / (ms_per_step * 1e-3)
 
@@ -311,25 +341,10 @@ def run_ours(args, w):
                 "peak_source": peaks["_source"] + " (sustained bf16 matmul; the kernel runs inside a long step)"}
 
     # end to end through the host-buffer C call: pinned host inputs, host outputs, copies inside
-    host = {n: t.cpu().pin_memory() for n, t in x.items()}
-    ho = sla.sla_prefill_host(handle, host["q_s"], host["q"], host["k"], host["v"], params)
-    n_e2e = max(2, min(args.steps, 5))
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    tt = time.perf_counter()
-    for _ in range(n_e2e):
-        sla.sla_prefill_host(handle, host["q_s"], host["q"], host["k"], host["v"], params,
-                             out=ho[0], lse=ho[1], anchor=ho[2], score=ho[3])
-    e2e_s = (time.perf_counter() - tt) / n_e2e
-    if dist:
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    h2d = sum(host[n].numel() * host[n].element_size() for n in ("q_s", "q", "k", "v"))
-    d2h = sum(t.numel() * t.element_size() for t in ho)
-    e2e = {"value": world * B * L / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-           "ms_per_step": e2e_s * 1e3}
+    host = None
+    if not (args.no_e2e and args.no_cpu_baseline):
+        host = {n: t.cpu().pin_memory() for n, t in x.items()}
+    e2e = None if args.no_e2e else measure_e2e(sla, handle, host, params, args, dist, dev, world, B, L)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -348,6 +363,8 @@ def run_ours(args, w):
         torch.cuda.empty_cache()
         dec = []
         for ci, steps in ((3, 256), (4, 128)):
+            if args.decode_only and args.decode_only != synth.CONFIGS[ci].name:
+                continue
             try:
                 dec.append(bench_decode(sla, handle, synth.CONFIGS[ci], steps if not args.quick else 16, peaks, dev))
             except torch.cuda.OutOfMemoryError as e:  # pragma: no cover
@@ -357,6 +374,7 @@ def run_ours(args, w):
         from oracle import sla_oracle as O
         rows = oracle_sample_rows(L, args.ref_rows)
         hn = {n: synth.to_numpy(t) for n, t in host.items()}
+        rows = rows[rows < L]
         secs = time_oracle_prefill(w, hn, rows)
         line["cpu_baseline"] = {"value": len(rows) * B / secs, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
                                 "sample": f"{len(rows)} evenly spaced query positions x all {Hq} heads, "
@@ -377,10 +395,15 @@ def main():
     ap.add_argument("--workload", type=int, default=1, help="index into the benchmark configurations (prefill ones)")
     ap.add_argument("--ref-rows", type=int, default=4096, help="query positions the CPU oracle is timed on")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--seq-len", type=int, default=0, help="shorter prefill sequence (for profiler captures)")
+    ap.add_argument("--decode-only", default="", help="decode_1M or decode_10M: only that decode loop besides the prefill part")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="short decode loops (for smoke runs)")
     args = ap.parse_args()
     w = synth.CONFIGS[args.workload]
+    if args.seq_len:
+        w = w.scaled(seq_len=args.seq_len, name=f"{w.name}_cut_to_{args.seq_len}")
     if w.kind != "prefill":
         raise SystemExit("--workload must name a prefill configuration; decode is reported alongside")
     if args.impl == "reference":
