@@ -307,13 +307,16 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
             if (tid < (ti.w & 0xff)) rec = p.recs[ti.z + tid];
             gather_q(tid < (ti.w & 0xff), rec.x);
         }
-        for (; tile < n_tiles; tile += tile_step, ++T) {
-            const int nblk = ti.w >> 8, sb0 = ti.y - nblk + 1, cnt = ti.w & 0xff;
-            const bool valid = tid < cnt;
-            // hand this tile's Q to the MMA issuer
+        // hands the gathered Q tile to the MMA issuer
+        auto publish_q = [&]() {
             ptx::cp_async_wait_all();
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(bar_q_full);
+        };
+        if (tile < n_tiles) publish_q();
+        for (; tile < n_tiles; tile += tile_step, ++T) {
+            const int nblk = ti.w >> 8, sb0 = ti.y - nblk + 1, cnt = ti.w & 0xff;
+            const bool valid = tid < cnt;
             // the next tile: its record is fetched now, its Q row during this tile's last key block
             const bool has_next = tile + tile_step < n_tiles;
             const int4 ti_next = has_next ? p.tiles[tile + tile_step] : make_int4(0, 0, 0, 0);
@@ -415,6 +418,9 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 ptx::tc_fence_before();
                 ptx::mbar_arrive(bar_p_ready + 8 * st);
             }
+            // the next tile's Q rows were requested a block ago: publish them now, so that its first
+            // S = Q K^T runs while this tile drains
+            if (ok && has_next) publish_q();
             // epilogue: normalised piece output and its log-sum-exp
             if (ok) ok = ptx::mbar_wait_warp(bar_o_full, T & 1u, abort_flag);
             if (!ok) break;
