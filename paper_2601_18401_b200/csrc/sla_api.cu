@@ -22,7 +22,9 @@ struct sla_handle_s {
 
 namespace {
 
-constexpr size_t kHeaderBytes = 256;
+// header of the workspace: status word at 0, completion counters of the decode step from byte 256
+constexpr size_t kHeaderBytes = 64 * 1024;
+constexpr size_t kCounterOffset = 256;
 
 sla_status_t fail(sla_handle_t h, sla_status_t code, const char *fmt, const char *detail = "") {
     if (h) snprintf(h->err, sizeof h->err, fmt, detail);
@@ -267,11 +269,14 @@ sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, con
     const sla::DecodePlan plan =
         sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim));
     if (plan.bytes + kHeaderBytes > h->ws_bytes) return fail(h, SLA_ERR_WORKSPACE, "workspace too small for this decode step%s");
-    if ((size_t)plan.n_anchor * sizeof(float) > 200 * 1024) return fail(h, SLA_ERR_UNSUPPORTED, "context too long for the decode top-k kernel%s");
+    if ((size_t)plan.n_anchor * sizeof(float) * 8 > 180 * 1024) return fail(h, SLA_ERR_UNSUPPORTED, "context too long for the decode top-k stage%s");
+    if ((size_t)(l->batch) * (l->n_kv_heads + l->n_q_heads) * sizeof(int) > kHeaderBytes - kCounterOffset)
+        return fail(h, SLA_ERR_UNSUPPORTED, "too many (batch, head) pairs for the decode step%s");
     cudaError_t e = sla::launch_decode(q_s, q, k_cache, v_cache, c, l->dtype, n_ctx, plan, h->ws + kHeaderBytes,
-                                       out, lse, out_anchor, out_score, static_cast<cudaStream_t>(stream));
+                                       reinterpret_cast<int *>(h->ws + kCounterOffset), out, lse, out_anchor,
+                                       out_score, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_decode_step");
-    h->launches += 4;
+    h->launches += 2;
     return SLA_OK;
 }
 

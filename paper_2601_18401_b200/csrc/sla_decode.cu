@@ -4,21 +4,25 @@
 // kernel spreads each head's tokens evenly over many CTAs (split-K), streams whole rows with 16-byte
 // loads, keeps a running (max, denominator, numerator) per lane group and merges at the end.
 //
-//   decode_score   grid (anchor chunks, B*Hkv, head tiles)   K anchor rows x G routing queries
-//   decode_topk    grid (B*Hq)                               k best anchors, spans, overlap clipping
-//   decode_attn    grid (n_splits, B*Hq)                     online softmax over an even token share
-//   decode_merge   grid (B*Hq)                               log-sum-exp merge of the split results
+//   decode_score   grid (anchor chunks, B*Hkv, head tiles)   K anchor rows x G routing queries; the CTA
+//                  that finishes a (batch, KV head) last selects the k best anchors of its G heads,
+//                  builds their spans and clips the overlaps
+//   decode_attn    grid (n_splits, B*Hq)                     online softmax over an even token share;
+//                  the CTA that finishes a head last merges the split results through their
+//                  log-sum-exp
+// "Last" is decided by an atomic counter per (batch, KV head) / per head in the handle's header
+// region; the last CTA puts the counter back to zero, so a step leaves them as it found them.
 #include <limits.h>
 #include <math_constants.h>
 
 #include "sla_kernels.h"
+#include "sla_topk.cuh"
 
 namespace sla {
 
 namespace {
 
 constexpr int kScoreThreads = 256;
-constexpr int kTopkThreads = 128;
 constexpr int kAttnThreads = 256;
 
 template <int LPR> __device__ inline float reduce_sub(float x) {
@@ -31,7 +35,10 @@ template <int LPR> __device__ inline float reduce_sub(float x) {
 template <typename T, int D, int GT>
 __global__ void __launch_bounds__(kScoreThreads)
 decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long long n_ctx, int n,
-             float *__restrict__ scores) {
+             float *__restrict__ scores, int *__restrict__ done, int *__restrict__ spans,
+             int32_t *__restrict__ out_anchor, float *__restrict__ out_score) {
+    extern __shared__ float dsm[];
+    __shared__ int s_last;
     constexpr int E = Vec16<T>::kElems;
     constexpr int LPR = D / E;
     constexpr int RPI = 32 / LPR;
@@ -75,94 +82,77 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
                 scores[((long long)b * c.Hq + h0 + t) * n + s] = tot * c.search_scale;
         }
     }
-}
 
-// ------------------------------------------------------------------------------------------------
-// Top-k of one head's anchor scores (largest first, smaller stride index on ties), the spans of the
-// selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)]) sorted and clipped to disjoint
-// pieces, and their cumulative token counts.
-__global__ void __launch_bounds__(kTopkThreads)
-decode_topk(Call c, long long n_ctx, int n, const float *__restrict__ scores, int *__restrict__ spans,
-            int32_t *__restrict__ out_anchor, float *__restrict__ out_score) {
-    extern __shared__ float sc[];
-    __shared__ float wv[kTopkThreads / 32];
-    __shared__ int ws[kTopkThreads / 32];
-    __shared__ int s_lo[kMaxTopK], s_hi[kMaxTopK], p_lo[kMaxTopK], p_hi[kMaxTopK];
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const long long bh = blockIdx.x;
-    const long long i = n_ctx - 1;
-    const float *src = scores + bh * n;
-    for (int s = tid; s < n; s += kTopkThreads) sc[s] = src[s];
+    // ---- the CTA that completes this (batch, KV head) selects and builds the spans
+    __threadfence();
     __syncthreads();
-
-    for (int j = 0; j < c.top_k; ++j) {
-        float bv = -CUDART_INF_F;
-        int bs = INT_MAX;
-        for (int s = tid; s < n; s += kTopkThreads) {
-            const float v = sc[s];
-            if (v > bv) { bv = v; bs = s; }
-        }
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-            const int os = __shfl_xor_sync(0xffffffffu, bs, off);
-            if (ov > bv || (ov == bv && os < bs)) { bv = ov; bs = os; }
-        }
-        if (lane == 0) { wv[warp] = bv; ws[warp] = bs; }
-        __syncthreads();
-        if (tid == 0) {
-            for (int w = 1; w < kTopkThreads / 32; ++w)
-                if (wv[w] > bv || (wv[w] == bv && ws[w] < bs)) { bv = wv[w]; bs = ws[w]; }
+    if (threadIdx.x == 0) {
+        const int total = gridDim.x * gridDim.z;
+        const int prev = atomicAdd(done + blockIdx.y, 1);
+        s_last = prev == total - 1;
+        if (s_last) done[blockIdx.y] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const int per_warp = n + 2 * topk::kCap + 4 * kMaxTopK;
+    float *sc = dsm + (size_t)warp * per_warp;
+    float *cand_v = sc + n;
+    int *cand_s = reinterpret_cast<int *>(cand_v + topk::kCap);
+    int *s_lo = cand_s + topk::kCap, *s_hi = s_lo + kMaxTopK, *p_lo = s_hi + kMaxTopK, *p_hi = p_lo + kMaxTopK;
+    const long long ell = base_len(i, c.span_len);
+    for (int hg = warp; hg < c.G; hg += kWarps) {
+        const long long bh = (long long)b * c.Hq + g * c.G + hg;
+        const float *src = scores + bh * n;
+        for (int s = lane; s < n; s += 32) sc[s] = __ldcg(src + s);   // written by other SMs: bypass L1
+        __syncwarp();
+        topk::select_topk(sc, n, c.top_k, i, cand_v, cand_s, out_anchor + bh * c.top_k, out_score + bh * c.top_k, lane);
+        // spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)]), sorted by
+        // (lo, hi) and clipped to disjoint pieces with their cumulative token counts
+        for (int j = lane; j < c.top_k; j += 32) {
+            const long long t = out_anchor[bh * c.top_k + j];
             int lo = INT_MAX, hi = -1;
-            if (bs != INT_MAX) {
-                const long long t = i + 1 - (long long)(bs + 1) * (bs + 1);
-                out_anchor[bh * c.top_k + j] = (int32_t)t;
-                out_score[bh * c.top_k + j] = bv;
-                sc[bs] = -CUDART_INF_F;
-                const long long ell = base_len(i, c.span_len);
+            if (t >= 0) {
                 const long long a = t - (long long)c.back * ell, z = t + (long long)c.fwd * ell;
                 lo = (int)(a > 0 ? a : 0);
                 hi = (int)(z < i ? z : i);
-            } else {
-                out_anchor[bh * c.top_k + j] = -1;
-                out_score[bh * c.top_k + j] = -CUDART_INF_F;
             }
             s_lo[j] = lo;
             s_hi[j] = hi;
         }
-        __syncthreads();
-    }
-    // rank sort by (lo, hi, index), then clip overlaps into disjoint pieces
-    if (tid < c.top_k) {
-        const int lo = s_lo[tid], hi = s_hi[tid];
-        int rank = 0;
-        for (int m = 0; m < c.top_k; ++m) {
-            const int lm = s_lo[m], hm = s_hi[m];
-            rank += (lm < lo) || (lm == lo && (hm < hi || (hm == hi && m < tid)));
-        }
-        p_lo[rank] = lo;
-        p_hi[rank] = hi;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int *start = spans + bh * (2 * c.top_k + 2);
-        int *cum = start + c.top_k;
-        int cnt = 0;
-        long long next_free = 0, total = 0;
-        cum[0] = 0;
-        for (int a = 0; a < c.top_k; ++a) {
-            const int lo = p_lo[a], hi = p_hi[a];
-            if (hi < 0) break;
-            const long long j0 = lo > next_free ? lo : next_free;
-            if (j0 <= hi) {
-                start[cnt] = (int)j0;
-                total += hi - j0 + 1;
-                cum[cnt + 1] = (int)total;
-                ++cnt;
+        __syncwarp();
+        for (int j = lane; j < c.top_k; j += 32) {
+            const int lo = s_lo[j], hi = s_hi[j];
+            int rank = 0;
+            for (int m = 0; m < c.top_k; ++m) {
+                const int lm = s_lo[m], hm = s_hi[m];
+                rank += (lm < lo) || (lm == lo && (hm < hi || (hm == hi && m < j)));
             }
-            if ((long long)hi + 1 > next_free) next_free = (long long)hi + 1;
+            p_lo[rank] = lo;
+            p_hi[rank] = hi;
         }
-        start[2 * c.top_k + 1] = cnt;
+        __syncwarp();
+        if (lane == 0) {
+            int *start = spans + bh * (2 * c.top_k + 2);
+            int *cum = start + c.top_k;
+            int cnt = 0;
+            long long next_free = 0, total = 0;
+            cum[0] = 0;
+            for (int a = 0; a < c.top_k; ++a) {
+                const int lo = p_lo[a], hi = p_hi[a];
+                if (hi < 0) break;
+                const long long j0 = lo > next_free ? lo : next_free;
+                if (j0 <= hi) {
+                    start[cnt] = (int)j0;
+                    total += hi - j0 + 1;
+                    cum[cnt + 1] = (int)total;
+                    ++cnt;
+                }
+                if ((long long)hi + 1 > next_free) next_free = (long long)hi + 1;
+            }
+            start[2 * c.top_k + 1] = cnt;
+        }
+        __syncwarp();
     }
 }
 
@@ -170,7 +160,9 @@ decode_topk(Call c, long long n_ctx, int n, const float *__restrict__ scores, in
 template <typename T, int D>
 __global__ void __launch_bounds__(kAttnThreads)
 decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, Call c,
-            const int *__restrict__ spans, float *__restrict__ partial) {
+            const int *__restrict__ spans, float *__restrict__ partial, int *__restrict__ done,
+            T *__restrict__ out, float *__restrict__ lse) {
+    __shared__ int s_last;
     constexpr int E = Vec16<T>::kElems;
     constexpr int LPR = D / E;
     constexpr int RPI = 32 / LPR;
@@ -303,32 +295,36 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
         if (tid == 0) { dst[0] = mm; dst[1] = ll; }
         dst[2 + tid] = aa;
     }
-}
-
-// ------------------------------------------------------------------------------------------------
-template <typename T, int D>
-__global__ void __launch_bounds__(D)
-decode_merge(Call c, int n_splits, const float *__restrict__ partial, T *__restrict__ out,
-             float *__restrict__ lse) {
-    const long long bh = blockIdx.x;
-    const int h = (int)(bh % c.Hq), b = (int)(bh / c.Hq), d = threadIdx.x;
-    const float *src = partial + bh * n_splits * (D + 2);
-    float mm = -CUDART_INF_F;
-    for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, src[s * (D + 2)]);
-    float ll = 0.f, aa = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const float ms = src[s * (D + 2)];
-        const float sc = (ms == -CUDART_INF_F) ? 0.f : exp2f(ms - mm);
-        ll += src[s * (D + 2) + 1] * sc;
-        aa += src[s * (D + 2) + 2 + d] * sc;
+    // ---- the CTA that completes this head merges the split results
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int prev = atomicAdd(done + bh, 1);
+        s_last = prev == n_splits - 1;
+        if (s_last) done[bh] = 0;
     }
-    out[b * c.q_sb + (long long)h * c.q_sh + d] = from_float<T>(ll > 0.f ? aa / ll : 0.f);
-    if (d == 0) lse[bh] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid < D) {
+        const float *src = partial + bh * n_splits * (D + 2);
+        float mm = -CUDART_INF_F;
+        for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, __ldcg(src + s * (D + 2)));
+        float ll = 0.f, aa = 0.f;
+        for (int s = 0; s < n_splits; ++s) {
+            const float ms = __ldcg(src + s * (D + 2));
+            const float sc = (ms == -CUDART_INF_F) ? 0.f : exp2f(ms - mm);
+            ll += __ldcg(src + s * (D + 2) + 1) * sc;
+            aa += __ldcg(src + s * (D + 2) + 2 + tid) * sc;
+        }
+        out[b * c.q_sb + (long long)h * c.q_sh + tid] = from_float<T>(ll > 0.f ? aa / ll : 0.f);
+        if (tid == 0) lse[bh] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
+    }
 }
 
 template <typename T, int D>
 cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const void *v, const Call &c,
-                          long long n_ctx, const DecodePlan &p, void *scratch, void *out, float *lse,
+                          long long n_ctx, const DecodePlan &p, void *scratch, int *counters, void *out, float *lse,
                           int32_t *out_anchor, float *out_score, cudaStream_t st) {
     constexpr int E = Vec16<T>::kElems;
     constexpr int RPI = 32 / (D / E);
@@ -336,33 +332,34 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
     float *scores = (float *)(base + p.off_scores);
     int *spans = (int *)(base + p.off_spans);
     float *partial = (float *)(base + p.off_partial);
+    int *done_bg = counters, *done_bh = counters + c.B * c.Hkv;
     const int n = p.n_anchor;
     const int rows_per_cta = (kScoreThreads / 32) * RPI * 2;
     const int gt = c.G % 8 == 0 ? 8 : c.G % 4 == 0 ? 4 : c.G % 2 == 0 ? 2 : 1;
     dim3 gs((n + rows_per_cta - 1) / rows_per_cta, c.B * c.Hkv, c.G / gt);
     const T *qs = (const T *)q_s, *kk = (const T *)k;
-    switch (gt) {
-        case 8: decode_score<T, D, 8><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, scores); break;
-        case 4: decode_score<T, D, 4><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, scores); break;
-        case 2: decode_score<T, D, 2><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, scores); break;
-        default: decode_score<T, D, 1><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, scores); break;
-    }
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    const size_t smem = (size_t)n * sizeof(float);
+    const size_t smem = (size_t)(kScoreThreads / 32) * (n + 2 * topk::kCap + 4 * kMaxTopK) * sizeof(float);
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
-    if (smem > 48 * 1024) {
-        e = cudaFuncSetAttribute(decode_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+#define SLA_LAUNCH_SCORE(GT)                                                                                         \
+    do {                                                                                                             \
+        auto kern = decode_score<T, D, GT>;                                                                          \
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        if (e == cudaSuccess)                                                                                        \
+            kern<<<gs, kScoreThreads, smem, st>>>(qs, kk, c, n_ctx, n, scores, done_bg, spans, out_anchor, out_score); \
+    } while (0)
+    switch (gt) {
+        case 8: SLA_LAUNCH_SCORE(8); break;
+        case 4: SLA_LAUNCH_SCORE(4); break;
+        case 2: SLA_LAUNCH_SCORE(2); break;
+        default: SLA_LAUNCH_SCORE(1); break;
     }
-    decode_topk<<<c.B * c.Hq, kTopkThreads, smem, st>>>(c, n_ctx, n, scores, spans, out_anchor, out_score);
+#undef SLA_LAUNCH_SCORE
+    if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     decode_attn<T, D><<<dim3(p.n_splits, c.B * c.Hq), kAttnThreads, 0, st>>>(
-        (const T *)q, kk, (const T *)v, c, spans, partial);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    decode_merge<T, D><<<c.B * c.Hq, D, 0, st>>>(c, p.n_splits, partial, (T *)out, lse);
+        (const T *)q, kk, (const T *)v, c, spans, partial, done_bh, (T *)out, lse);
     return cudaGetLastError();
 }
 
@@ -408,14 +405,14 @@ DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots) {
 }
 
 cudaError_t launch_decode(const void *q_s, const void *q, const void *k, const void *v, const Call &c,
-                          int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, void *out,
-                          float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st) {
+                          int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, int *counters,
+                          void *out, float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st) {
     if (dtype == SLA_F32) {
-        return c.D == 64 ? decode_launch<float, 64>(q_s, q, k, v, c, n_ctx, plan, scratch, out, lse, out_anchor, out_score, st)
-                         : decode_launch<float, 128>(q_s, q, k, v, c, n_ctx, plan, scratch, out, lse, out_anchor, out_score, st);
+        return c.D == 64 ? decode_launch<float, 64>(q_s, q, k, v, c, n_ctx, plan, scratch, counters, out, lse, out_anchor, out_score, st)
+                         : decode_launch<float, 128>(q_s, q, k, v, c, n_ctx, plan, scratch, counters, out, lse, out_anchor, out_score, st);
     }
-    return c.D == 64 ? decode_launch<__nv_bfloat16, 64>(q_s, q, k, v, c, n_ctx, plan, scratch, out, lse, out_anchor, out_score, st)
-                     : decode_launch<__nv_bfloat16, 128>(q_s, q, k, v, c, n_ctx, plan, scratch, out, lse, out_anchor, out_score, st);
+    return c.D == 64 ? decode_launch<__nv_bfloat16, 64>(q_s, q, k, v, c, n_ctx, plan, scratch, counters, out, lse, out_anchor, out_score, st)
+                     : decode_launch<__nv_bfloat16, 128>(q_s, q, k, v, c, n_ctx, plan, scratch, counters, out, lse, out_anchor, out_score, st);
 }
 
 }  // namespace sla

@@ -57,8 +57,9 @@ struct DecodePlan {
 // cta_slots = SM count x resident decode_attn CTAs per SM (see decode_attn_blocks_per_sm)
 DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots);
 int decode_attn_blocks_per_sm(int dtype, int D);
+// counters: B*Hkv + B*Hq ints, zero on entry and zero again on exit (completion counters)
 cudaError_t launch_decode(const void *q_s, const void *q, const void *k, const void *v, const Call &c,
-                          int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, void *out,
-                          float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st);
+                          int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, int *counters,
+                          void *out, float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st);
 
 }  // namespace sla

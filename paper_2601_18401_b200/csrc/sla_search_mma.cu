@@ -17,6 +17,7 @@
 #include <math_constants.h>
 
 #include "sla_kernels.h"
+#include "sla_topk.cuh"
 
 namespace sla {
 
@@ -24,12 +25,8 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 constexpr int kWarps = 8;
-constexpr int kCap = 64;   // candidate slots per warp in the selection
-
-__device__ __forceinline__ uint32_t order_key(float x) {
-    const uint32_t u = __float_as_uint(x);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
+using topk::kCap;
+using topk::select_topk;
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -37,89 +34,6 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// Top-k of sc[0..n) for one head; writes anchors/scores.  All lanes of the warp take part.
-__device__ void select_topk(float *sc, int n, int top_k, long long i, float *cand_v, int *cand_s,
-                            int32_t *out_anchor, float *out_score, int lane) {
-    const uint32_t kNegInfKey = order_key(-CUDART_INF_F);
-    // A. lane maxima over the strided slots
-    float lm = -CUDART_INF_F;
-    for (int s = lane; s < n; s += 32) lm = fmaxf(lm, sc[s]);
-    // B. threshold = top_k-th largest lane maximum (there are at least top_k scores >= it)
-    uint32_t cur = order_key(lm), tau_key = kNegInfKey;
-    if (n > top_k && top_k <= 32) {
-        for (int j = 0; j < top_k; ++j) {
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, cur);
-            tau_key = mx;
-            if (mx == kNegInfKey) break;
-            const uint32_t who = __ballot_sync(0xffffffffu, cur == mx);
-            if (lane == __ffs(who) - 1) cur = kNegInfKey;
-        }
-    }
-    // C. compact the candidates >= threshold
-    int count = 0;
-    for (int s0 = 0; s0 < n; s0 += 32) {
-        const int s = s0 + lane;
-        const float v = s < n ? sc[s] : 0.f;
-        const bool take = s < n && order_key(v) >= tau_key;
-        const uint32_t mask = __ballot_sync(0xffffffffu, take);
-        if (take) {
-            const int pos = count + __popc(mask & ((1u << lane) - 1u));
-            if (pos < kCap) { cand_v[pos] = v; cand_s[pos] = s; }
-        }
-        count += __popc(mask);
-    }
-    __syncwarp();
-    if (count <= kCap) {
-        // D. k rounds of warp arg-max over the candidates (two per lane)
-        float v0 = lane < count ? cand_v[lane] : -CUDART_INF_F, v1 = lane + 32 < count ? cand_v[lane + 32] : -CUDART_INF_F;
-        int s0 = lane < count ? cand_s[lane] : INT_MAX, s1 = lane + 32 < count ? cand_s[lane + 32] : INT_MAX;
-        for (int j = 0; j < top_k; ++j) {
-            const bool first = v0 > v1 || (v0 == v1 && s0 <= s1);
-            const float bv = first ? v0 : v1;
-            const int bs = first ? s0 : s1;
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, order_key(bv));
-            const int smin = __reduce_min_sync(0xffffffffu, (order_key(bv) == mx && bs != INT_MAX) ? bs : INT_MAX);
-            if (smin == INT_MAX) {   // fewer candidates than slots: pad
-                if (lane == 0) { out_anchor[j] = -1; out_score[j] = -CUDART_INF_F; }
-                continue;
-            }
-            if (bs == smin && order_key(bv) == mx) {
-                out_anchor[j] = (int32_t)(i + 1 - (long long)(bs + 1) * (bs + 1));
-                out_score[j] = bv;
-                if (first) { v0 = -CUDART_INF_F; s0 = INT_MAX; } else { v1 = -CUDART_INF_F; s1 = INT_MAX; }
-            }
-        }
-    } else {
-        // many equal scores at the threshold: plain k rounds over all scores
-        for (int j = 0; j < top_k; ++j) {
-            float bv = -CUDART_INF_F;
-            int bs = INT_MAX;
-            for (int s = lane; s < n; s += 32) {
-                const float v = sc[s];
-                if (v > bv) { bv = v; bs = s; }
-            }
-#pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-                const int os = __shfl_xor_sync(0xffffffffu, bs, off);
-                if (ov > bv || (ov == bv && os < bs)) { bv = ov; bs = os; }
-            }
-            if (lane == 0) {
-                if (bs != INT_MAX) {
-                    out_anchor[j] = (int32_t)(i + 1 - (long long)(bs + 1) * (bs + 1));
-                    out_score[j] = bv;
-                    sc[bs] = -CUDART_INF_F;
-                } else {
-                    out_anchor[j] = -1;
-                    out_score[j] = -CUDART_INF_F;
-                }
-            }
-            __syncwarp();
-        }
-    }
-    __syncwarp();
 }
 
 __global__ void __launch_bounds__(kWarps * 32)
