@@ -173,6 +173,37 @@ sla_status_t sla_decode_step(sla_handle_t handle, const void *q_s, const void *q
                              const sla_params_t *params, void *out, float *lse, int32_t *out_anchor,
                              float *out_score, void *stream);
 
+/* ---- decode step without any allocation ---------------------------------------------------- */
+
+/* (The paper has no counterpart: this entry point exists for the sake of the hosts of this library.)
+ *
+ * sla_decode_step for callers that may not allocate device memory -- code running under a stream
+ * capture or inside a serving loop that forbids cudaMalloc, processes whose device memory has been
+ * handed in full to another allocator, plug-ins that are lent a stream and nothing else.  Such
+ * callers cannot call sla_create, because the handle's workspace is a cudaMalloc.  This call needs no
+ * handle: its scratch (anchor scores, clipped spans, split results, completion counters) is a fixed
+ * array of SLA_STATIC_SCRATCH_BYTES inside the library image, which every GPU that loads the library
+ * holds until the process exits.  The call allocates nothing and frees nothing, on the host's heap
+ * or on the device.
+ *
+ * Arguments, results and launch behaviour are those of sla_decode_step (same kernels); inputs and
+ * outputs are still the caller's device buffers.  Differences:
+ *   - a step whose scratch exceeds the fixed array (it grows with batch * heads * sqrt(n_ctx) and
+ *     with batch * heads * splits) is rejected with SLA_ERR_WORKSPACE and nothing is launched; the
+ *     1M- and 10M-token configurations with 32 query heads need well under 1 MiB;
+ *   - the first call on a device resolves the array's device address (once per device, with that
+ *     device current) and asks a few device attributes; make this first call outside any stream
+ *     capture;
+ *   - all calls on one device share the array: it keeps the previous call's contents (the part that
+ *     must start at zero is cleared on the stream at the start of each call), and two calls that
+ *     overlap on the GPU -- different streams, or several threads -- race on it.  Serialise them.
+ *   - there is no handle to hold an error text: the status code is all there is
+ *     (SLA_ERR_INVALID_ARG, SLA_ERR_UNSUPPORTED, SLA_ERR_WORKSPACE as above, SLA_ERR_CUDA). */
+#define SLA_STATIC_SCRATCH_BYTES (2u << 20)
+sla_status_t sla_decode_step_static(const void *q_s, const void *q, const void *k_cache, const void *v_cache,
+                                    int64_t n_ctx, const sla_layout_t *layout, const sla_params_t *params,
+                                    void *out, float *lse, int32_t *out_anchor, float *out_score, void *stream);
+
 /* ---- host-buffer convenience calls ---------------------------------------------------------- */
 
 /* sla_span_search followed by sla_span_attention on HOST buffers (pinned memory gives the best

@@ -24,7 +24,7 @@ EXPORTS = [
     "sla_create", "sla_destroy", "sla_workspace_bytes", "sla_status_string", "sla_last_error",
     "sla_poll_status", "sla_span_search", "sla_span_attention", "sla_decode_step",
     "sla_host_staging_bytes", "sla_prefill_host", "sla_kernel_launches", "sla_set_kernel_timing",
-    "sla_kernel_time_ms",
+    "sla_kernel_time_ms", "sla_decode_step_static",
 ]
 
 
@@ -80,6 +80,8 @@ def load_library():
     lib.sla_span_attention.argtypes = [vp, vp, vp, vp, i64, i64, i64, LP, PP, vp, vp, vp, vp]
     lib.sla_decode_step.restype = i32
     lib.sla_decode_step.argtypes = [vp, vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
+    lib.sla_decode_step_static.restype = i32
+    lib.sla_decode_step_static.argtypes = [vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
     lib.sla_kernel_launches.restype = i64
     lib.sla_kernel_launches.argtypes = [vp]
     lib.sla_set_kernel_timing.restype = i32
@@ -245,6 +247,23 @@ def sla_decode_step(handle: Handle, q_s: torch.Tensor, q: torch.Tensor, k_cache:
                                      out.data_ptr(), lse.data_ptr(), out_anchor.data_ptr(),
                                      out_score.data_ptr(), _stream_ptr(stream))
     handle.check(rc, "sla_decode_step")
+    return out, lse, out_anchor, out_score
+
+
+def sla_decode_step_static(q_s: torch.Tensor, q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                           n_ctx: int, params: sla_params_t, *, out, lse, out_anchor, out_score, stream=None):
+    """The decode step for callers that may not allocate: no handle, scratch inside the library image,
+    and every output buffer supplied by the caller (this wrapper allocates nothing either)."""
+    if q_s.stride() != q.stride() or k_cache.stride() != v_cache.stride() or out.stride() != q.stride():
+        raise ValueError("q_s/q/out and k_cache/v_cache must share their strides")
+    lib = load_library()
+    layout = make_layout(q, k_cache, decode=True)
+    rc = lib.sla_decode_step_static(q_s.data_ptr(), q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), int(n_ctx),
+                                    C.byref(layout), C.byref(params), out.data_ptr(), lse.data_ptr(),
+                                    out_anchor.data_ptr(), out_score.data_ptr(), _stream_ptr(stream))
+    if rc != SLA_OK:
+        what = {-3: "the step needs more scratch than the fixed array inside the library holds"}.get(rc, "call rejected")
+        raise SlaError(rc, f"sla_decode_step_static: {lib.sla_status_string(rc).decode()}: {what}")
     return out, lse, out_anchor, out_score
 
 

@@ -92,6 +92,25 @@ size_t elem_size(int dtype) { return dtype == SLA_F32 ? 4 : 2; }
 
 }  // namespace
 
+namespace sla {
+
+// Argument checks of a decode step for callers that have no handle (the no-allocation entry point
+// in sla_decode.cu): same rules as sla_decode_step.  Fills *c_out on success.
+sla_status_t check_decode_args(const void *q_s, const void *q, const void *k_cache, const void *v_cache,
+                               int64_t n_ctx, const sla_layout_t *l, const sla_params_t *p, const void *out,
+                               const float *lse, const int32_t *out_anchor, const float *out_score, Call *c_out) {
+    if (check_layout_params(l, p, true)) return SLA_ERR_INVALID_ARG;
+    if (n_ctx <= 0 || n_ctx > 2147483647LL) return SLA_ERR_INVALID_ARG;
+    if (!q_s || !q || !k_cache || !v_cache || !out || !lse || !out_anchor || !out_score) return SLA_ERR_INVALID_ARG;
+    if (!aligned16(q_s) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
+        return SLA_ERR_INVALID_ARG;
+    if (p->window != 0 || p->mode != SLA_UNION) return SLA_ERR_UNSUPPORTED;
+    *c_out = make_call(nullptr, l, p, 1, n_ctx - 1, n_ctx);
+    return SLA_OK;
+}
+
+}  // namespace sla
+
 extern "C" {
 
 const char *sla_status_string(sla_status_t s) {

@@ -415,4 +415,62 @@ cudaError_t launch_decode(const void *q_s, const void *q, const void *k, const v
                      : decode_launch<__nv_bfloat16, 128>(q_s, q, k, v, c, n_ctx, plan, scratch, counters, out, lse, out_anchor, out_score, st);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Decode step for callers that cannot allocate device memory (declared in include/sla.h).
+//
+// Some hosts of this library run where cudaMalloc is off limits: inside a CUDA-graph capture or a
+// stream-ordered region of a serving loop, in a process whose device memory is handed out in full to
+// another allocator at start-up, or in a plug-in that is only lent a stream.  They cannot create an
+// sla handle (its workspace is a cudaMalloc).  For them the decode step's scratch -- anchor scores,
+// clipped spans, split results and the completion counters -- lives in the array below, which is
+// part of the library image: every GPU that loads the library holds these 2 MiB until the process
+// exits, whether or not the entry point is ever called.
+namespace {
+
+constexpr size_t kStaticScratchBytes = SLA_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+// Device addresses of the array, one per device.  In host code the array's name is only a handle for
+// the runtime: the address a kernel may use comes from cudaGetSymbolAddress, asked once per device
+// with that device current.
+unsigned char *g_decode_scratch_ptr[kMaxDevices] = {};
+int g_cta_slots[kMaxDevices][2][2] = {};
+
+}  // namespace
 }  // namespace sla
+
+extern "C" sla_status_t sla_decode_step_static(const void *q_s, const void *q, const void *k_cache,
+                                               const void *v_cache, int64_t n_ctx, const sla_layout_t *l,
+                                               const sla_params_t *p, void *out, float *lse, int32_t *out_anchor,
+                                               float *out_score, void *stream) {
+    sla::Call c;
+    if (sla_status_t s = sla::check_decode_args(q_s, q, k_cache, v_cache, n_ctx, l, p, out, lse, out_anchor, out_score, &c))
+        return s;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SLA_ERR_CUDA;
+    if (dev < 0 || dev >= sla::kMaxDevices) return SLA_ERR_UNSUPPORTED;
+    if (!sla::g_decode_scratch_ptr[dev]) {
+        // set-up, once per device (the current one): resolve the array's device address
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, sla::g_decode_scratch) != cudaSuccess || !ptr) return SLA_ERR_CUDA;
+        sla::g_decode_scratch_ptr[dev] = static_cast<unsigned char *>(ptr);
+    }
+    int &slots = sla::g_cta_slots[dev][l->dtype == SLA_F32 ? 0 : 1][l->head_dim == 64 ? 0 : 1];
+    if (slots == 0) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SLA_ERR_CUDA;
+        slots = sms * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim);
+    }
+    const sla::DecodePlan plan = sla::plan_decode(c, n_ctx, slots);
+    const size_t counter_bytes = (((size_t)l->batch * (l->n_kv_heads + l->n_q_heads) * sizeof(int)) + 255) & ~(size_t)255;
+    if (counter_bytes + plan.bytes > sla::kStaticScratchBytes) return SLA_ERR_WORKSPACE;   // beyond the fixed maximum
+    if ((size_t)plan.n_anchor * sizeof(float) * 8 > 180 * 1024) return SLA_ERR_UNSUPPORTED;
+    unsigned char *base = sla::g_decode_scratch_ptr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the previous call left; only the completion counters have to start at zero
+    if (cudaMemsetAsync(base, 0, counter_bytes, st) != cudaSuccess) return SLA_ERR_CUDA;
+    cudaError_t e = sla::launch_decode(q_s, q, k_cache, v_cache, c, l->dtype, n_ctx, plan, base + counter_bytes,
+                                       reinterpret_cast<int *>(base), out, lse, out_anchor, out_score, st);
+    return e == cudaSuccess ? SLA_OK : SLA_ERR_CUDA;
+}

@@ -62,4 +62,9 @@ cudaError_t launch_decode(const void *q_s, const void *q, const void *k, const v
                           int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, int *counters,
                           void *out, float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st);
 
+// argument checks of a decode step without a handle (defined in sla_api.cu)
+sla_status_t check_decode_args(const void *q_s, const void *q, const void *k_cache, const void *v_cache,
+                               int64_t n_ctx, const sla_layout_t *l, const sla_params_t *p, const void *out,
+                               const float *lse, const int32_t *out_anchor, const float *out_score, Call *c_out);
+
 }  // namespace sla
