@@ -111,6 +111,15 @@ __device__ __forceinline__ unsigned long long fadd2(unsigned long long a, unsign
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// A shared-memory matrix descriptor moved forward by `bytes` (the start address sits in the low word
+// in units of 16 bytes, and the window is far below the field's range, so no carry leaves it).
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) {
+    uint32_t lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(desc));
+    lo += bytes >> 4;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(desc) : "r"(lo), "r"(hi));
+    return desc;
+}
 __device__ __forceinline__ float ex2_approx(float x) {
 #ifdef SLA_EXP_NOMUFU
     return fmaf(x, 1e-3f, 1.f);
@@ -223,6 +232,9 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
         uint32_t n_kv = 0, T = 0;
         int tile = blockIdx.x;
         int nblk = tile < n_tiles ? (p.tiles[tile].w >> 8) : 0;
+        const uint64_t desc_q0 = ptx::smem_desc_sw128(base + kOffQ, 16, 1024);
+        const uint64_t desc_k0 = ptx::smem_desc_sw128(base + kOffK, 16, 1024);
+        const uint64_t desc_v0 = ptx::smem_desc_sw128(base + kOffV, kKVBytes / 2, 1024);
         for (; tile < n_tiles; tile += tile_step, ++T) {
             const int nblk_next = tile + tile_step < n_tiles ? (p.tiles[tile + tile_step].w >> 8) : 0;
             bool ok = ptx::mbar_wait(bar_q_full, T & 1u, abort_flag);
@@ -236,12 +248,12 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                     if (ptx::mbar_test_wait(bar_k_full + 8 * ks, (n / kKS) & 1u)) {
                         ptx::tc_fence_after();
                         const uint32_t d_s = tmem + kColS + sbuf * kBK;
+                        const uint64_t dk = desc_advance(desc_k0, ks * kKVBytes);
 #pragma unroll
                         for (int kk = 0; kk < kD / 16; ++kk) {
                             const uint32_t half = kk >> 2, inner = (kk & 3) * 32;
-                            const uint64_t da = ptx::smem_desc_sw128(base + kOffQ + half * (kQBytes / 2) + inner, 16, 1024);
-                            const uint64_t db = ptx::smem_desc_sw128(base + kOffK + ks * kKVBytes + half * (kKVBytes / 2) + inner, 16, 1024);
-                            ptx::mma_ss(d_s, da, db, kIdescS, kk > 0);
+                            ptx::mma_ss(d_s, desc_advance(desc_q0, half * (kQBytes / 2) + inner),
+                                        desc_advance(dk, half * (kKVBytes / 2) + inner), kIdescS, kk > 0);
                         }
                         ptx::mma_commit(bar_s_full + 8 * sbuf);
                         ptx::mma_commit(bar_k_empty + 8 * ks);
@@ -255,11 +267,11 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                     if (o_free && ptx::mbar_test_wait(bar_p_ready + 8 * vs, ph) && ptx::mbar_test_wait(bar_v_full + 8 * vs, ph)) {
                         ptx::tc_fence_after();
                         const uint32_t a_p = tmem + kColS + vs * kBK;   // P aliases S: 64 bf16 = 32 columns
+                        const uint64_t dv = desc_advance(desc_v0, vs * kKVBytes);
 #pragma unroll
-                        for (int kk = 0; kk < kBK / 16; ++kk) {
-                            const uint64_t db = ptx::smem_desc_sw128(base + kOffV + vs * kKVBytes + kk * 2048, kKVBytes / 2, 1024);
-                            ptx::mma_ts(tmem + kColO, a_p + kk * 8, db, kIdescO, (ipv > 0 || kk > 0) ? 1u : 0u);
-                        }
+                        for (int kk = 0; kk < kBK / 16; ++kk)
+                            ptx::mma_ts(tmem + kColO, a_p + kk * 8, desc_advance(dv, kk * 2048), kIdescO,
+                                        (ipv > 0 || kk > 0) ? 1u : 0u);
                         ptx::mma_commit(bar_v_empty + 8 * vs);
                         if (ipv == nblk - 1) ptx::mma_commit(bar_o_full);
                         ++ipv;
@@ -346,13 +358,15 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 float bm = -CUDART_INF_F;
                 if (any) {
                     if (!full) {
+                        // bit c of the mask: column c of the block lies inside the piece
+                        const int ca = lo > k0 ? lo - k0 : 0, cb = hi - k0 < kBK - 1 ? hi - k0 : kBK - 1;
+                        const unsigned long long inside = (~0ull >> (63 - (cb - ca))) << ca;
+                        const uint32_t in2[2] = {static_cast<uint32_t>(inside), static_cast<uint32_t>(inside >> 32)};
 #pragma unroll
                         for (int hlf = 0; hlf < 2; ++hlf)
 #pragma unroll
-                            for (int cc = 0; cc < 32; ++cc) {
-                                const int kp = k0 + hlf * 32 + cc;
-                                if (kp < lo || kp > hi) sr[hlf][cc] = 0xff800000u;   // -inf
-                            }
+                            for (int cc = 0; cc < 32; ++cc)
+                                if (!(in2[hlf] & (1u << cc))) sr[hlf][cc] = 0xff800000u;   // -inf
                     }
                     float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
@@ -374,7 +388,7 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                     if (!ok) break;
                     ptx::tc_fence_after();
                     const float f = need ? ex2_approx(m_ref - bm) : 1.f;
-#pragma unroll
+#pragma unroll 1
                     for (int q4 = 0; q4 < 4; ++q4) {
                         uint32_t o[32];
                         ptx::tmem_ld32(lane_addr + kColO + q4 * 32, o);
@@ -430,7 +444,7 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 const long long slot = (long long)rec.x * p.top_k + rec.y;
                 __half *dst = p.part_o + slot * kD;
                 uint32_t exps = 0;   // biased exponent of each 32-column chunk's largest magnitude
-#pragma unroll
+#pragma unroll 1
                 for (int q4 = 0; q4 < 4; ++q4) {
                     uint32_t o[32];
                     ptx::tmem_ld32(lane_addr + kColO + q4 * 32, o);
