@@ -129,6 +129,24 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// Gathers one Q row (256 B) into the swizzled A-operand layout with 16-byte async copies; a null
+// source zero-fills the row.  Kept out of line: it runs once per tile from two places, and the
+// kernel's hot loop is faster the less code surrounds it.
+__device__ __noinline__ void gather_q_row(const bf16 *src, uint8_t *q_tile, uint32_t q_row, int tid) {
+    if (src) {
+#pragma unroll
+        for (int cidx = 0; cidx < 16; ++cidx) {
+            const uint32_t dst = q_row + (cidx >> 3) * (kQBytes / 2) + (((cidx & 7) ^ (tid & 7)) << 4);
+            ptx::cp_async16(dst, src + cidx * 8);
+        }
+    } else {
+        uint4 *qdst = reinterpret_cast<uint4 *>(q_tile);
+#pragma unroll
+        for (int cidx = 0; cidx < 16; ++cidx)
+            qdst[(cidx >> 3) * (kQBytes / 32) + tid * 8 + (cidx & 7)] = make_uint4(0, 0, 0, 0);
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 2)
 tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -293,23 +311,14 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
         // ---------------- row threads: Q gather, softmax per key block, epilogue
         const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
         const uint32_t q_row = base + kOffQ + tid * 128;
-        // Gathers one Q row (256 B) into the swizzled A-operand layout with 16-byte async copies.
         auto gather_q = [&](bool row_valid, int row) {
+            const bf16 *src = nullptr;
             if (row_valid) {
                 const int rc = row % p.Lc, bh = row / p.Lc;
                 const int h = bh % p.Hq, bb = bh / p.Hq;
-                const bf16 *src = p.q + bb * p.q_sb + h * p.q_sh + (p.r0 + rc) * p.q_st;
-#pragma unroll
-                for (int cidx = 0; cidx < 16; ++cidx) {
-                    const uint32_t dst = q_row + (cidx >> 3) * (kQBytes / 2) + (((cidx & 7) ^ (tid & 7)) << 4);
-                    ptx::cp_async16(dst, src + cidx * 8);
-                }
-            } else {
-                uint4 *qdst = reinterpret_cast<uint4 *>(smem + kOffQ);
-#pragma unroll
-                for (int cidx = 0; cidx < 16; ++cidx)
-                    qdst[(cidx >> 3) * (kQBytes / 32) + tid * 8 + (cidx & 7)] = make_uint4(0, 0, 0, 0);
+                src = p.q + bb * p.q_sb + h * p.q_sh + (p.r0 + rc) * p.q_st;
             }
+            gather_q_row(src, smem + kOffQ, q_row, tid);
         };
         uint32_t n_kv = 0, T = 0;
         int tile = blockIdx.x;
@@ -353,21 +362,20 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 ptx::tmem_wait_ld();
                 const int k0 = (sb0 + j) * kBK;
                 const bool any = valid && k0 <= hi && k0 + kBK - 1 >= lo;
-                const bool full = any && k0 >= lo && k0 + kBK - 1 <= hi;
+                if (!(any && k0 >= lo && k0 + kBK - 1 <= hi)) {
+                    // bit c of the mask: column c of the block lies inside the piece
+                    const int ca = lo > k0 ? lo - k0 : 0, cb = hi - k0 < kBK - 1 ? hi - k0 : kBK - 1;
+                    const unsigned long long inside = any ? (~0ull >> (63 - (cb - ca))) << ca : 0ull;
+                    const uint32_t in2[2] = {static_cast<uint32_t>(inside), static_cast<uint32_t>(inside >> 32)};
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf)
+#pragma unroll
+                        for (int cc = 0; cc < 32; ++cc)
+                            if (!(in2[hlf] & (1u << cc))) sr[hlf][cc] = 0xff800000u;   // -inf
+                }
                 // block maximum on the raw logits (softmax_scale > 0 on this path), four independent chains
-                float bm = -CUDART_INF_F;
-                if (any) {
-                    if (!full) {
-                        // bit c of the mask: column c of the block lies inside the piece
-                        const int ca = lo > k0 ? lo - k0 : 0, cb = hi - k0 < kBK - 1 ? hi - k0 : kBK - 1;
-                        const unsigned long long inside = (~0ull >> (63 - (cb - ca))) << ca;
-                        const uint32_t in2[2] = {static_cast<uint32_t>(inside), static_cast<uint32_t>(inside >> 32)};
-#pragma unroll
-                        for (int hlf = 0; hlf < 2; ++hlf)
-#pragma unroll
-                            for (int cc = 0; cc < 32; ++cc)
-                                if (!(in2[hlf] & (1u << cc))) sr[hlf][cc] = 0xff800000u;   // -inf
-                    }
+                float bm;
+                {
                     float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
                     for (int hlf = 0; hlf < 2; ++hlf)
@@ -401,9 +409,11 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 }
                 if (first && bm > -CUDART_INF_F) m_ref = bm;   // first keys of this row
                 uint32_t pk[32];
-                if (any && bm > -CUDART_INF_F) {
-                    // p = 2^(s*scale - m_ref), two columns per packed fp32x2 instruction
-                    const unsigned long long sc2 = pack2(p.scale2, p.scale2), nm2 = pack2(-m_ref, -m_ref);
+                {
+                    // p = 2^(s*scale - m_ref), two columns per packed fp32x2 instruction; masked columns
+                    // hold -inf and give 0 (a row with no key so far has m_ref = -inf: it subtracts 0)
+                    const float neg_m = m_ref > -CUDART_INF_F ? -m_ref : 0.f;
+                    const unsigned long long sc2 = pack2(p.scale2, p.scale2), nm2 = pack2(neg_m, neg_m);
                     unsigned long long acc2[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) acc2[u] = pack2(0.f, 0.f);
@@ -423,9 +433,6 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                     unpack2(fadd2(acc2[0], acc2[1]), s0, s1);
                     unpack2(fadd2(acc2[2], acc2[3]), s2, s3);
                     l += (s0 + s1) + (s2 + s3);
-                } else {
-#pragma unroll
-                    for (int cc = 0; cc < 32; ++cc) pk[cc] = 0u;
                 }
                 ptx::tmem_st32(s_addr, pk);
                 ptx::tmem_wait_st();
