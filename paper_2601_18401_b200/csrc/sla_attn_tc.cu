@@ -44,7 +44,7 @@ using bf16 = __nv_bfloat16;
 constexpr int kD = 128;
 using tc::kBK;    // keys per block
 using tc::kRows;  // pieces per tile
-constexpr int kThreads = 192;
+constexpr int kThreads = 192;   // 4 row warps, MMA issuer, TMA producer
 constexpr int kTmemCols = 256;
 constexpr uint32_t kColS = 0;    // S buffers at columns 0 and 64
 constexpr uint32_t kColO = 128;
@@ -166,7 +166,7 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
     const uint32_t bar_s_full = ptx::smem_u32(&meta->s_full[0]), bar_p_ready = ptx::smem_u32(&meta->p_ready[0]);
 
     if (tid == 0) {
-        ptx::mbar_init(bar_q_full, kRows);
+        ptx::mbar_init(bar_q_full, 4);   // one arrival per row warp
         ptx::mbar_init(bar_o_full, 1);
         ptx::mbar_init(bar_o_empty, 4);
         for (int s = 0; s < kKS; ++s) {
@@ -177,7 +177,7 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
             ptx::mbar_init(bar_v_full + 8 * s, 1);
             ptx::mbar_init(bar_v_empty + 8 * s, 1);
             ptx::mbar_init(bar_s_full + 8 * s, 1);
-            ptx::mbar_init(bar_p_ready + 8 * s, kRows);
+            ptx::mbar_init(bar_p_ready + 8 * s, 4);
         }
         meta->abort_flag = 0;
         ptx::fence_barrier_init();
@@ -205,42 +205,64 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
     const int tile_step = gridDim.x;
 
     if (warp == 5 && lane == 0) {
-        // ---------------- TMA producer: K(j) then V(j) of every key block, as far ahead as the stages allow
-        uint32_t n_kv = 0;
-        int tile = blockIdx.x;
-        int4 ti = tile < n_tiles ? p.tiles[tile] : make_int4(0, 0, 0, 0);
-        for (; tile < n_tiles; tile += tile_step) {
-            const int nblk = ti.w >> 8, sb0 = ti.y - nblk + 1;
+        // ---------------- TMA producer, event driven: the K blocks and the V blocks of the CTA's tile
+        // sequence are two independent streams, each running as far ahead as its own stages allow (a
+        // K stage frees when its S = Q K^T is done, long before the V stage of the same block).
+        struct Cursor {
+            int tile, j, nblk, sb0, ch, cb;
+            uint32_t n;
+        };
+        auto open_tile = [&](Cursor &cu) {
+            if (cu.tile < n_tiles) {
+                const int4 ti = p.tiles[cu.tile];
+                cu.nblk = ti.w >> 8;
+                cu.sb0 = ti.y - cu.nblk + 1;
+                cu.ch = ti.x % p.Hkv;
+                cu.cb = ti.x / p.Hkv;
+                cu.j = 0;
+            }
+        };
+        auto issue = [&](Cursor &cu, const CUtensorMap *tm, uint32_t bar_full, uint32_t dst) {
             int c[4];
-            c[1 + p.slot_h] = ti.x % p.Hkv;
-            c[1 + p.slot_b] = ti.x / p.Hkv;
-            const int4 ti_next = tile + tile_step < n_tiles ? p.tiles[tile + tile_step] : make_int4(0, 0, 0, 0);
-            bool ok = true;
-            for (int j = 0; j < nblk; ++j) {
-                const uint32_t n = n_kv + j;
-                c[1 + p.slot_t] = (sb0 + j) * kBK;
-                {
-                    const uint32_t st = n % kKS, ph = (n / kKS) & 1u;
-                    ok = ptx::mbar_wait(bar_k_empty + 8 * st, ph ^ 1u, abort_flag);
-                    if (!ok) break;
-                    ptx::mbar_arrive_expect_tx(bar_k_full + 8 * st, kKVBytes);
-                    const uint32_t dst = base + kOffK + st * kKVBytes;
-                    ptx::tma_load_4d(dst, &tm_k, bar_k_full + 8 * st, 0, c[1], c[2], c[3]);
-                    ptx::tma_load_4d(dst + kKVBytes / 2, &tm_k, bar_k_full + 8 * st, 64, c[1], c[2], c[3]);
-                }
-                {
-                    const uint32_t st = n % kVS, ph = (n / kVS) & 1u;
-                    ok = ptx::mbar_wait(bar_v_empty + 8 * st, ph ^ 1u, abort_flag);
-                    if (!ok) break;
-                    ptx::mbar_arrive_expect_tx(bar_v_full + 8 * st, kKVBytes);
-                    const uint32_t dst = base + kOffV + st * kKVBytes;
-                    ptx::tma_load_4d(dst, &tm_v, bar_v_full + 8 * st, 0, c[1], c[2], c[3]);
-                    ptx::tma_load_4d(dst + kKVBytes / 2, &tm_v, bar_v_full + 8 * st, 64, c[1], c[2], c[3]);
+            c[1 + p.slot_h] = cu.ch;
+            c[1 + p.slot_b] = cu.cb;
+            c[1 + p.slot_t] = (cu.sb0 + cu.j) * kBK;
+            ptx::mbar_arrive_expect_tx(bar_full, kKVBytes);
+            ptx::tma_load_4d(dst, tm, bar_full, 0, c[1], c[2], c[3]);
+            ptx::tma_load_4d(dst + kKVBytes / 2, tm, bar_full, 64, c[1], c[2], c[3]);
+            ++cu.n;
+            if (++cu.j == cu.nblk) {
+                cu.tile += tile_step;
+                open_tile(cu);
+            }
+        };
+        Cursor ck{(int)blockIdx.x, 0, 0, 0, 0, 0, 0u}, cv{(int)blockIdx.x, 0, 0, 0, 0, 0, 0u};
+        open_tile(ck);
+        cv = ck;
+        uint32_t idle = 0;
+        while (cv.tile < n_tiles) {
+            bool progressed = false;
+            if (ck.tile < n_tiles) {
+                const uint32_t st = ck.n % kKS;
+                if (ptx::mbar_test_wait(bar_k_empty + 8 * st, ((ck.n / kKS) & 1u) ^ 1u)) {
+                    issue(ck, &tm_k, bar_k_full + 8 * st, base + kOffK + st * kKVBytes);
+                    progressed = true;
                 }
             }
-            if (!ok) break;
-            n_kv += nblk;
-            ti = ti_next;
+            {
+                const uint32_t st = cv.n % kVS;
+                if (cv.n < ck.n &&   // K first: V(n) is never requested before K(n)
+                    ptx::mbar_test_wait(bar_v_empty + 8 * st, ((cv.n / kVS) & 1u) ^ 1u)) {
+                    issue(cv, &tm_v, bar_v_full + 8 * st, base + kOffV + st * kKVBytes);
+                    progressed = true;
+                }
+            }
+            if (progressed) {
+                idle = 0;
+            } else if (__nanosleep(40), ++idle > ptx::kSpinLimit || ((idle & 63u) == 0u && *abort_flag)) {
+                *abort_flag = 1;
+                break;
+            }
         }
     } else if (warp == 4 && lane == 0) {
         // ---------------- MMA issuer, event driven: S(j) as soon as K(j) has landed and an S buffer
@@ -332,7 +354,8 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
         auto publish_q = [&]() {
             ptx::cp_async_wait_all();
             ptx::fence_proxy_async_smem();
-            ptx::mbar_arrive(bar_q_full);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar_q_full);
         };
         if (tile < n_tiles) publish_q();
         for (; tile < n_tiles; tile += tile_step, ++T) {
@@ -437,7 +460,8 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 ptx::tmem_st32(s_addr, pk);
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before();
-                ptx::mbar_arrive(bar_p_ready + 8 * st);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar_p_ready + 8 * st);
             }
             // the next tile's Q rows were requested a block ago: publish them now, so that its first
             // S = Q K^T runs while this tile drains
@@ -451,11 +475,8 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                 const long long slot = (long long)rec.x * p.top_k + rec.y;
                 __half *dst = p.part_o + slot * kD;
                 uint32_t exps = 0;   // biased exponent of each 32-column chunk's largest magnitude
-#pragma unroll 1
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint32_t o[32];
-                    ptx::tmem_ld32(lane_addr + kColO + q4 * 32, o);
-                    ptx::tmem_wait_ld();
+                // one 32-column chunk: block exponent, fp16 mantissas, two 32-byte stores
+                auto emit = [&](uint32_t (&o)[32], int q4) {
                     if (valid) {
                         float amax = 0.f;
 #pragma unroll
@@ -480,14 +501,28 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
                             ptx::st_global_v8(dst + q4 * 32 + s8 * 16, w);
                         }
                     }
-                }
+                };
+                // the TMEM read of the next chunk is in flight while this one is converted and stored
+                uint32_t oa[32], ob[32];
+                ptx::tmem_ld32(lane_addr + kColO, oa);
+                ptx::tmem_wait_ld();
+                ptx::tmem_ld32(lane_addr + kColO + 32, ob);
+                emit(oa, 0);
+                ptx::tmem_wait_ld();
+                ptx::tmem_ld32(lane_addr + kColO + 64, oa);
+                emit(ob, 1);
+                ptx::tmem_wait_ld();
+                ptx::tmem_ld32(lane_addr + kColO + 96, ob);
+                emit(oa, 2);
+                ptx::tmem_wait_ld();
+                // O is in registers: the next tile's first PV may overwrite it
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar_o_empty);
+                emit(ob, 3);
                 if (valid)
                     p.part_lse[slot] = make_float2(l > 0.f ? m_ref + log2f(l) : -CUDART_INF_F, __uint_as_float(exps));
             }
-            // O has been read: the next tile's first PV may overwrite it
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar_o_empty);
             n_kv += nblk;
             rec = rec_next;
             ti = ti_next;

@@ -46,6 +46,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // raises the CTA's abort flag and returns false.  Nothing in the kernels waits without a bound.
 constexpr uint32_t kSpinLimit = 1u << 22;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+#pragma unroll 1
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 31u) == 31u && *abort_flag) return false;
@@ -56,6 +57,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // Warp-collective form: every lane of a converged warp waits on the same barrier and all lanes
 // return the same answer, so that the .sync.aligned TMEM instructions that follow stay convergent.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+#pragma unroll 1
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         const bool done = mbar_try_wait(bar, parity);
         if (__all_sync(0xffffffffu, done)) return true;
@@ -72,6 +74,9 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 }
 
 // ---- TMA ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void prefetch_l2(const void *ptr) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
 __device__ __forceinline__ void prefetch_tensormap(const void *tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
