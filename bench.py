@@ -36,9 +36,9 @@ from paper_2601_18401_b200 import synth
 
 METRIC = "prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one tc_attend launch, from the ncu capture summarised
-# in profiles/ (taken on a quarter-length case and scaled by the number of tiles); None until measured
-TC_ATTEND_DRAM_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one tc_attend launch of the default workload
+# (L = 65536), from the one-pass ncu capture of the full-size launch summarised in profiles/
+TC_ATTEND_DRAM_BYTES_PER_LAUNCH = {65536: 7.52e9, 16384: 1.43e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -333,7 +333,7 @@ def run_ours(args, w):
     peak_tf = peaks["bf16_tflops_sustained"]
     roofline = {"bound": "tensor", "kernel": "tc_attend (tcgen05 span-attention)" if kern_n else "attn_rows_simt",
                 "achieved": tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": tflops / peak_tf,
-                "traffic": TC_ATTEND_DRAM_BYTES_PER_LAUNCH if kern_n else None,
+                "traffic": TC_ATTEND_DRAM_BYTES_PER_LAUNCH.get(L) if kern_n else None,
                 "flops_per_launch": flops, "ms_per_launch": kern_ms, "launches_timed": kern_n,
                 "whole_call": {"sla_span_attention_ms": attn_ms, "sla_span_search_ms": ms_per_step - attn_ms,
                                "attention_tflops": flops / (attn_ms * 1e-3) / 1e12,
