@@ -66,10 +66,10 @@ typedef enum {
 
 typedef enum { SLA_F32 = 0, SLA_BF16 = 1 } sla_dtype_t;
 
-/* SLA_UNION: one softmax over the de-duplicated union of the selected spans (reduces to dense
- * causal attention when the selection covers every key).  SLA_PER_SPAN (Algorithm 1 literally: one
- * softmax per span, then the softmax gate of Section "Combination") is not implemented yet and
- * returns SLA_ERR_UNSUPPORTED. */
+/* SLA_UNION: one softmax over the de-duplicated union of the selected spans and the local window
+ * (reduces to dense causal attention when the selection covers every key); sla_span_attention and
+ * sla_decode_step.  SLA_PER_SPAN: Algorithm 1 literally, one softmax per selected span united with
+ * the window, then the softmax gate of Section "Combination"; sla_span_attention_gated. */
 typedef enum { SLA_UNION = 0, SLA_PER_SPAN = 1 } sla_mode_t;
 
 typedef struct sla_handle_s *sla_handle_t; /* opaque; owns the device workspace */
@@ -92,8 +92,9 @@ typedef struct {
     int32_t span_len;     /* l > 0: fixed base span length; 0: l(i) = ceil(sqrt(i)) (Algorithm 1)  */
     int32_t back_factor;  /* b >= 0; b >= 2 is needed for full coverage (Section "Span attention") */
     int32_t fwd_factor;   /* f >= 0                                                               */
-    int32_t window;       /* local window w of Algorithm 1; only 0 is implemented                 */
-    int32_t mode;         /* sla_mode_t; only SLA_UNION is implemented                            */
+    int32_t window;       /* local window w of Algorithm 1: W = [max(0,i-w+1), i]; 0 = none;
+                             anchors inside W are no candidates (decode step: only 0)           */
+    int32_t mode;         /* sla_mode_t (decode step: only SLA_UNION)                             */
     float search_scale;   /* multiplies the search score (the paper's equation has none: 1.0f)    */
     float softmax_scale;  /* multiplies the attention logits ("scaled dot-product": 1/sqrt(D))     */
 } sla_params_t;
@@ -159,6 +160,19 @@ sla_status_t sla_span_attention(sla_handle_t handle, const void *q, const void *
                                 int64_t Lq, int64_t q_pos0, int64_t Lkv, const sla_layout_t *layout,
                                 const sla_params_t *params, const int32_t *anchor, void *out,
                                 float *lse, void *stream);
+
+/* Algorithm 1 literally (params->mode = SLA_PER_SPAN): for every selected anchor t one softmax over
+ * J_t = S_t united with the window W (A_t), then O = sum_t alpha_t A_t with alpha = softmax of the
+ * search scores of the selected anchors (Section "Combination"); a row without a valid anchor attends
+ * to W alone (out = 0, lse = -inf when there is no window either).
+ *   score      in   [B, Hq, Lq, top_k] fp32, contiguous, device: the scores sla_span_search returned
+ *   lse        out  [B, Hq, Lq] fp32: log-sum-exp of the first (best-scoring) selected span
+ *   lse_span   out  [B, Hq, Lq, top_k] fp32 or NULL: log-sum-exp of every J_t, -inf for padding
+ * Other arguments, layouts and errors as for sla_span_attention. */
+sla_status_t sla_span_attention_gated(sla_handle_t handle, const void *q, const void *k, const void *v,
+                                      int64_t Lq, int64_t q_pos0, int64_t Lkv, const sla_layout_t *layout,
+                                      const sla_params_t *params, const int32_t *anchor, const float *score,
+                                      void *out, float *lse, float *lse_span, void *stream);
 
 /* ---- decode step (Section "Kernel design", "Decoding path") -------------------------------- */
 

@@ -24,7 +24,7 @@ EXPORTS = [
     "sla_create", "sla_destroy", "sla_workspace_bytes", "sla_status_string", "sla_last_error",
     "sla_poll_status", "sla_span_search", "sla_span_attention", "sla_decode_step",
     "sla_host_staging_bytes", "sla_prefill_host", "sla_kernel_launches", "sla_set_kernel_timing",
-    "sla_kernel_time_ms", "sla_decode_step_static",
+    "sla_kernel_time_ms", "sla_decode_step_static", "sla_span_attention_gated",
 ]
 
 
@@ -78,6 +78,8 @@ def load_library():
     lib.sla_span_search.argtypes = [vp, vp, vp, i64, i64, i64, LP, PP, vp, vp, vp]
     lib.sla_span_attention.restype = i32
     lib.sla_span_attention.argtypes = [vp, vp, vp, vp, i64, i64, i64, LP, PP, vp, vp, vp, vp]
+    lib.sla_span_attention_gated.restype = i32
+    lib.sla_span_attention_gated.argtypes = [vp, vp, vp, vp, i64, i64, i64, LP, PP, vp, vp, vp, vp, vp, vp]
     lib.sla_decode_step.restype = i32
     lib.sla_decode_step.argtypes = [vp, vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
     lib.sla_decode_step_static.restype = i32
@@ -227,6 +229,31 @@ def sla_span_attention(handle: Handle, q: torch.Tensor, k: torch.Tensor, v: torc
                                         anchor.data_ptr(), out.data_ptr(), lse.data_ptr(), _stream_ptr(stream))
     handle.check(rc, "sla_span_attention")
     return out, lse
+
+
+def sla_span_attention_gated(handle: Handle, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
+                             anchor: torch.Tensor, score: torch.Tensor, params: sla_params_t, *,
+                             q_pos0: int = 0, Lkv: Optional[int] = None, out=None, lse=None, lse_span=None,
+                             stream=None):
+    """Per-span softmax and gate (params.mode = SLA_PER_SPAN): anchor int32 and score fp32 [B,Hq,Lq,k]
+    -> out (q's dtype and strides), lse fp32 [B,Hq,Lq], lse_span fp32 [B,Hq,Lq,k]."""
+    B, Hq, Lq, D = q.shape
+    Lkv = k.shape[2] if Lkv is None else int(Lkv)
+    assert anchor.dtype == torch.int32 and anchor.is_contiguous() and anchor.shape[:3] == (B, Hq, Lq)
+    assert score.dtype == torch.float32 and score.is_contiguous() and score.shape == anchor.shape
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty(B, Hq, Lq, dtype=torch.float32, device=q.device)
+    if lse_span is None:
+        lse_span = torch.empty(anchor.shape, dtype=torch.float32, device=q.device)
+    layout = make_layout(q, k)
+    rc = handle._lib.sla_span_attention_gated(handle.ptr, q.data_ptr(), k.data_ptr(), v.data_ptr(), Lq,
+                                              int(q_pos0), Lkv, C.byref(layout), C.byref(params),
+                                              anchor.data_ptr(), score.data_ptr(), out.data_ptr(),
+                                              lse.data_ptr(), lse_span.data_ptr(), _stream_ptr(stream))
+    handle.check(rc, "sla_span_attention_gated")
+    return out, lse, lse_span
 
 
 def sla_decode_step(handle: Handle, q_s: torch.Tensor, q: torch.Tensor, k_cache: torch.Tensor,

@@ -57,13 +57,15 @@ const char *check_layout_params(const sla_layout_t *l, const sla_params_t *p, bo
     if (p->top_k < 1 || p->top_k > sla::kMaxTopK) return "top_k must be in 1..64";
     if (p->span_len < 0 || p->back_factor < 0 || p->fwd_factor < 0) return "span_len and factors must be >= 0";
     if (p->window < 0) return "window must be >= 0";
+    if (p->mode != SLA_UNION && p->mode != SLA_PER_SPAN) return "mode must be SLA_UNION or SLA_PER_SPAN";
     if (!(p->softmax_scale == p->softmax_scale) || !(p->search_scale == p->search_scale)) return "scale is NaN";
     return nullptr;
 }
 
-sla_status_t check_supported(sla_handle_t h, const sla_params_t *p) {
-    if (p->window != 0) return fail(h, SLA_ERR_UNSUPPORTED, "window > 0 is not implemented%s");
-    if (p->mode != SLA_UNION) return fail(h, SLA_ERR_UNSUPPORTED, "only SLA_UNION is implemented%s");
+// The decode step implements the union mode without a window only.
+sla_status_t check_supported_decode(sla_handle_t h, const sla_params_t *p) {
+    if (p->window != 0) return fail(h, SLA_ERR_UNSUPPORTED, "window > 0 is not implemented for the decode step%s");
+    if (p->mode != SLA_UNION) return fail(h, SLA_ERR_UNSUPPORTED, "only SLA_UNION is implemented for the decode step%s");
     return SLA_OK;
 }
 
@@ -76,6 +78,7 @@ sla::Call make_call(const sla_handle_t h, const sla_layout_t *l, const sla_param
     c.kv_sb = l->kv_stride_b; c.kv_sh = l->kv_stride_h; c.kv_st = l->kv_stride_t;
     c.Lq = Lq; c.q_pos0 = q_pos0; c.Lkv = Lkv;
     c.top_k = p->top_k; c.span_len = p->span_len; c.back = p->back_factor; c.fwd = p->fwd_factor;
+    c.window = p->window; c.mode = p->mode;
     c.search_scale = p->search_scale; c.softmax_scale = p->softmax_scale;
     c.status = h ? reinterpret_cast<int *>(h->ws) : nullptr;
     return c;
@@ -229,7 +232,6 @@ sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int
     if (const char *why = check_prefill_range(Lq, q_pos0, Lkv)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!q_s || !k || !out_anchor || !out_score) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
     if (!aligned16(q_s) || !aligned16(k)) return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
-    if (sla_status_t s = check_supported(h, p)) return s;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!h->force_simt && sla::search_mma_supported(c, l->dtype)) {
@@ -243,16 +245,17 @@ sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int
     return SLA_OK;
 }
 
-sla_status_t sla_span_attention(sla_handle_t h, const void *q, const void *k, const void *v, int64_t Lq,
-                                int64_t q_pos0, int64_t Lkv, const sla_layout_t *l, const sla_params_t *p,
-                                const int32_t *anchor, void *out, float *lse, void *stream) {
-    if (!h) return SLA_ERR_INVALID_ARG;
-    if (const char *why = check_layout_params(l, p, false)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+namespace {
+
+// Body of the two span-attention entry points (score and lse_span are NULL in the union mode).
+sla_status_t span_attention_impl(sla_handle_t h, const void *q, const void *k, const void *v, int64_t Lq,
+                                 int64_t q_pos0, int64_t Lkv, const sla_layout_t *l, const sla_params_t *p,
+                                 const int32_t *anchor, const float *score, void *out, float *lse,
+                                 float *lse_span, void *stream, const char *what) {
     if (const char *why = check_prefill_range(Lq, q_pos0, Lkv)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!q || !k || !v || !anchor || !out || !lse) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
         return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
-    if (sla_status_t s = check_supported(h, p)) return s;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!h->force_simt && sla::tc_attention_supported(c, l->dtype)) {
@@ -260,16 +263,41 @@ sla_status_t sla_span_attention(sla_handle_t h, const void *q, const void *k, co
         const long long min_chunk = Lq < 1024 ? Lq : 1024;
         const sla::TcPlan probe = sla::plan_attention_tc(c, (int)min_chunk);
         if (probe.ok && probe.bytes <= h->scratch_avail) {
-            cudaError_t e = sla::launch_attn_tc(q, k, v, c, anchor, out, lse, h->ws + kHeaderBytes,
+            cudaError_t e = sla::launch_attn_tc(q, k, v, c, anchor, score, out, lse, lse_span, h->ws + kHeaderBytes,
                                                 h->scratch_avail, h->sm_count, st, &h->launches, &h->timer);
-            if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_attention (tensor-core path)");
+            if (e != cudaSuccess) return cuda_fail(h, e, what);
             return SLA_OK;
         }
     }
-    cudaError_t e = sla::launch_attn_simt(q, k, v, c, l->dtype, anchor, out, lse, st);
-    if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_attention");
+    cudaError_t e = sla::launch_attn_simt(q, k, v, c, l->dtype, anchor, score, out, lse, lse_span, st);
+    if (e != cudaSuccess) return cuda_fail(h, e, what);
     h->launches += 1;
     return SLA_OK;
+}
+
+}  // namespace
+
+sla_status_t sla_span_attention(sla_handle_t h, const void *q, const void *k, const void *v, int64_t Lq,
+                                int64_t q_pos0, int64_t Lkv, const sla_layout_t *l, const sla_params_t *p,
+                                const int32_t *anchor, void *out, float *lse, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (const char *why = check_layout_params(l, p, false)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (p->mode != SLA_UNION)
+        return fail(h, SLA_ERR_INVALID_ARG, "SLA_PER_SPAN needs the search scores: call sla_span_attention_gated%s");
+    return span_attention_impl(h, q, k, v, Lq, q_pos0, Lkv, l, p, anchor, nullptr, out, lse, nullptr, stream,
+                               "sla_span_attention");
+}
+
+sla_status_t sla_span_attention_gated(sla_handle_t h, const void *q, const void *k, const void *v, int64_t Lq,
+                                      int64_t q_pos0, int64_t Lkv, const sla_layout_t *l,
+                                      const sla_params_t *p, const int32_t *anchor, const float *score,
+                                      void *out, float *lse, float *lse_span, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (const char *why = check_layout_params(l, p, false)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (p->mode != SLA_PER_SPAN) return fail(h, SLA_ERR_INVALID_ARG, "sla_span_attention_gated needs mode = SLA_PER_SPAN%s");
+    if (!score) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
+    return span_attention_impl(h, q, k, v, Lq, q_pos0, Lkv, l, p, anchor, score, out, lse, lse_span, stream,
+                               "sla_span_attention_gated");
 }
 
 sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, const void *k_cache,
@@ -283,7 +311,7 @@ sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, con
         return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
     if (!aligned16(q_s) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
         return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
-    if (sla_status_t s = check_supported(h, p)) return s;
+    if (sla_status_t s = check_supported_decode(h, p)) return s;
     sla::Call c = make_call(h, l, p, 1, n_ctx - 1, n_ctx);
     const sla::DecodePlan plan =
         sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim));

@@ -650,6 +650,7 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 bool tc_attention_shape_ok(const Call &c, int dtype) {
     if (dtype != SLA_BF16 || c.D != kD) return false;
+    if (c.window != 0 || c.mode != SLA_UNION) return false;
     if (c.kv_st < kD || c.top_k > kMaxTopK || !(c.softmax_scale > 0.f)) return false;
     const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
     const long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
@@ -694,7 +695,7 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
 }
 
 cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor,
-                           void *out, float *lse, void *scratch, size_t scratch_bytes, int sm_count,
+                           const float *score, void *out, float *lse, float *lse_span, void *scratch, size_t scratch_bytes, int sm_count,
                            cudaStream_t st, long long *launches, KernelTimer *timer) {
     // the largest chunk of query positions whose scratch fits
     long long Lc = c.Lq;

@@ -22,6 +22,7 @@ struct Call {
     long long kv_sb, kv_sh, kv_st;  // strides of k / v, in elements
     long long Lq, q_pos0, Lkv;
     int top_k, span_len, back, fwd;
+    int window, mode;               // local window w (0 = none); sla_mode_t
     float search_scale, softmax_scale;
     int *status;                    // device status word
 };

@@ -9,7 +9,8 @@ namespace sla {
 cudaError_t launch_search_simt(const void *q_s, const void *k, const Call &c, int dtype,
                                int32_t *out_anchor, float *out_score, cudaStream_t st);
 cudaError_t launch_attn_simt(const void *q, const void *k, const void *v, const Call &c, int dtype,
-                             const int32_t *anchor, void *out, float *lse, cudaStream_t st);
+                             const int32_t *anchor, const float *score, void *out, float *lse, float *lse_span,
+                             cudaStream_t st);
 
 // Optional device-side timing of the dominant kernel of a call (CUDA events on the caller's stream).
 struct KernelTimer {
@@ -40,8 +41,8 @@ bool tc_attention_supported(const Call &c, int dtype); // shape test + driver en
 TcPlan plan_attention_tc(const Call &c, int Lc);
 // Splits the query rows into chunks whose scratch fits `scratch_bytes`; adds its kernel launches to
 // *launches.  Returns cudaErrorMemoryAllocation when not even one query position fits.
-cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor,
-                           void *out, float *lse, void *scratch, size_t scratch_bytes, int sm_count,
+cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor, const float *score,
+                           void *out, float *lse, float *lse_span, void *scratch, size_t scratch_bytes, int sm_count,
                            cudaStream_t st, long long *launches, KernelTimer *timer);
 
 // ---- decode step (sla_decode.cu) ---------------------------------------------------------------

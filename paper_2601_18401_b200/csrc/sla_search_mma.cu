@@ -102,7 +102,7 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
 }  // namespace
 
 bool search_mma_supported(const Call &c, int dtype) {
-    if (dtype != SLA_BF16 || c.D != 128) return false;
+    if (dtype != SLA_BF16 || c.D != 128 || c.window != 0) return false;
     const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
     const int heads = c.G < 8 ? c.G : 8;
     return (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float) <= 200 * 1024;

@@ -1,0 +1,91 @@
+"""GPU parity of the two output modes and the local window (Algorithm 1: W = [max(0, i-w+1), i],
+anchors inside W are no candidates, J_t = S_t united with W; Section "Combination": the softmax gate
+over the selected anchors' search scores) against the oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import parity_util as P
+from oracle import sla_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sla():
+    import paper_2601_18401_b200 as sla_pkg
+    return sla_pkg
+
+
+@pytest.fixture(scope="module")
+def handle(sla):
+    h = sla.Handle(0, 256 << 20)
+    yield h
+    h.close()
+
+
+def workload(**kw):
+    from paper_2601_18401_b200 import synth
+    base = synth.Workload("modes", "prefill", 1, 4, 2, 128, 1111, "bf16", 16, 4, seed=77)
+    return base.scaled(**kw)
+
+
+def run_modes(sla, handle, w, window, q_pos0=0):
+    from paper_2601_18401_b200 import synth
+    x = synth.make_prefill(w, device="cuda:0")
+    L = w.seq_len
+    q_s, q = x["q_s"][:, :, q_pos0:], x["q"][:, :, q_pos0:]
+    host = P.host_inputs({"q_s": q_s, "q": q, "k": x["k"], "v": x["v"]})
+    code = synth.dtype_code(w.dtype)
+    # search: anchors inside the window are excluded
+    pu = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, window=window, head_dim=w.head_dim)
+    anchor, score = sla.sla_span_search(handle, q_s, x["k"], pu, q_pos0=q_pos0)
+    torch.cuda.synchronize()
+    ref_s = O.span_search(host["q_s"], host["k"], code, top_k=w.top_k, q_pos0=q_pos0, window=window)
+    P.compare_search(anchor, score, ref_s, q_pos0=q_pos0)
+    a_host = np.ascontiguousarray(anchor.cpu().numpy())
+    inside = (a_host >= 0) & (a_host > (np.arange(q_pos0, L)[None, None, :, None] - window))
+    assert not inside.any(), "an anchor inside the window was selected"
+    kw = dict(span_len=w.span_len, back_factor=w.back_factor, fwd_factor=w.fwd_factor, window=window,
+              q_pos0=q_pos0)
+    # union mode: one softmax over spans and window
+    out, lse = sla.sla_span_attention(handle, q, x["k"], x["v"], anchor, pu, q_pos0=q_pos0)
+    torch.cuda.synchronize()
+    ref_u = O.span_attention(host["q"], host["k"], host["v"], code, a_host, mode=O.UNION, **kw)
+    P.compare_attention(out, lse, ref_u, w.dtype)
+    # per-span mode with the gate, on the GPU's own scores
+    pg = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, window=window,
+                         mode=sla.SLA_PER_SPAN, head_dim=w.head_dim)
+    out_g, lse_g, lse_span = sla.sla_span_attention_gated(handle, q, x["k"], x["v"], anchor, score, pg,
+                                                         q_pos0=q_pos0)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    ref_g = O.span_attention(host["q"], host["k"], host["v"], code, a_host, mode=O.PER_SPAN,
+                             score=score.cpu().numpy().astype(np.float64), **kw)
+    P.compare_attention(out_g, lse_g, ref_g, w.dtype)
+    ls = lse_span.cpu().numpy().astype(np.float64)
+    fin = np.isfinite(ref_g["lse_span"])
+    assert np.array_equal(np.isneginf(ls), ~fin)
+    assert not fin.any() or np.abs(ls[fin] - ref_g["lse_span"][fin]).max() <= P.LSE_TOL[w.dtype]
+    return dict(out=out, out_g=out_g, anchor=anchor)
+
+
+@pytest.mark.parametrize("window", [0, 8, 48, 300])
+@pytest.mark.parametrize("kw", [
+    dict(),                                                        # bf16 D128 GQA (tensor-core shapes)
+    dict(dtype="f32", head_dim=64, n_q_heads=2, n_kv_heads=1, seq_len=700),
+    dict(span_len=0, back_factor=4, fwd_factor=2, top_k=2),        # the paper's kernel settings
+    dict(top_k=40, seq_len=300, span_len=5),                       # padding; rows with nothing selected
+])
+def test_modes_and_window(sla, handle, kw, window):
+    run_modes(sla, handle, workload(**kw), window)
+
+
+def test_chunked_prefill_with_window(sla, handle):
+    run_modes(sla, handle, workload(seq_len=1500), 100, q_pos0=900)
+
+
+def test_single_anchor_modes_agree(sla, handle):
+    """With top_k = 1 the gate is 1 and both modes compute the same attention."""
+    r = run_modes(sla, handle, workload(top_k=1, span_len=40), 24)
+    assert torch.equal(r["out"], r["out_g"])

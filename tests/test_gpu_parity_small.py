@@ -157,8 +157,8 @@ def test_error_returns(sla, handle):
     w = workload(seq_len=64)
     x = synth.make_prefill(w, device="cuda:0")
     with pytest.raises(sla.SlaError) as e:
-        sla.sla_span_search(handle, x["q_s"], x["k"], sla.make_params(4, 16, window=8))
-    assert e.value.status == -2
+        sla.sla_span_search(handle, x["q_s"], x["k"], sla.make_params(4, 16, window=-8))
+    assert e.value.status == -1
     with pytest.raises(sla.SlaError) as e:
         sla.sla_span_search(handle, x["q_s"], x["k"], sla.make_params(0, 16))
     assert e.value.status == -1
@@ -169,7 +169,7 @@ def test_error_returns(sla, handle):
         sla.sla_span_attention(handle, x["q"], x["k"], x["v"],
                                torch.zeros(1, 4, 64, 4, dtype=torch.int32, device="cuda"),
                                sla.make_params(4, 16, mode=sla.SLA_PER_SPAN))
-    assert e.value.status == -2
+    assert e.value.status == -1   # the gate needs the scores: sla_span_attention_gated
     small = sla.Handle(0, 1024)
     kc = torch.zeros(1, 2, 100000, 128, dtype=torch.bfloat16, device="cuda")
     qq = torch.zeros(1, 4, 128, dtype=torch.bfloat16, device="cuda")
