@@ -44,14 +44,14 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
     for (int x = threadIdx.x; x < nk; x += kPrepThreads) hist[x] = 0;
     __syncthreads();
 
-    int lo[kMaxTopK], hi[kMaxTopK];
+    int lo[kMaxTopK + 1], hi[kMaxTopK + 1], slot[kMaxTopK + 1];
     // sub-pass A: this CTA's pieces per bucket
     for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
         const int hg = (int)(q / a.Lc), rc = (int)(q % a.Lc);
         const int h = g * a.G + hg;
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
         const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
-        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len), a.back, a.fwd, lo, hi, a.status);
+        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len), a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
         if (PASS == 0) a.n_pieces[((long long)b * a.Hq + h) * a.Lc + rc] = (unsigned char)cnt;
         for (int j = 0; j < cnt; ++j) atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
     }
@@ -72,11 +72,11 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
         const int h = g * a.G + hg;
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
         const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
-        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len), a.back, a.fwd, lo, hi, a.status);
+        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len), a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
         const int row = (int)(((long long)b * a.Hq + h) * a.Lc + rc);
         for (int j = 0; j < cnt; ++j) {
             const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
-            a.recs[pos] = make_int4(row, j, lo[j], hi[j]);
+            a.recs[pos] = make_int4(row, slot[j], lo[j], hi[j]);
         }
     }
     }

@@ -72,16 +72,16 @@ static_assert(sizeof(Meta) <= kMetaBytes, "meta block too large");
 struct TcParams {
     const bf16 *q;
     long long q_sb, q_sh, q_st;
-    int Hq, G, Lc, top_k;
+    int Hq, G, Lc, slots;      // slots: partial results per row (top_k, + 1 with a local window)
     long long r0;              // first query row of the chunk
     float scale2;              // softmax_scale * log2(e)
     int slot_t, slot_h, slot_b;  // positions of (token, head, batch) among tensor-map coordinates 1..3
     const int4 *recs;          // sorted piece records {row, j, lo, hi}
     const int4 *tiles;         // {b*Hkv+g, end block, first record, record count | key blocks to walk << 8}
     const int *n_tiles;
-    __half *part_o;            // [rows*top_k][128] normalised piece outputs, fp16 with one power-of-two
+    __half *part_o;            // [rows*slots][128] normalised piece outputs, fp16 with one power-of-two
                                // scale per 32-column chunk (block floating point)
-    float2 *part_lse;          // [rows*top_k] {log2-domain log-sum-exp of the piece, four chunk exponents}
+    float2 *part_lse;          // [rows*slots] {log2-domain log-sum-exp of the piece, four chunk exponents}
     int *status;
     int Hkv;
 };
@@ -472,7 +472,7 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
             ptx::tc_fence_after();
             {
                 const float inv = l > 0.f ? 1.f / l : 0.f;
-                const long long slot = (long long)rec.x * p.top_k + rec.y;
+                const long long slot = (long long)rec.x * p.slots + rec.y;
                 __half *dst = p.part_o + slot * kD;
                 uint32_t exps = 0;   // biased exponent of each 32-column chunk's largest magnitude
                 // one 32-column chunk: block exponent, fp16 mantissas, two 32-byte stores
@@ -548,15 +548,15 @@ tc_attend(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUte
 // Per row: merge the normalised piece outputs through their log-sum-exp.  16 threads per row.
 __global__ void __launch_bounds__(256)
 tc_merge(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
-         const unsigned char *__restrict__ n_pieces, Call c, int Lc, long long r0, bf16 *__restrict__ out,
-         float *__restrict__ lse) {
+         const unsigned char *__restrict__ n_pieces, Call c, int slots, int Lc, long long r0,
+         bf16 *__restrict__ out, float *__restrict__ lse) {
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long row = gid >> 4;
     const int sub = (int)(gid & 15);
     const long long rows = (long long)c.B * c.Hq * Lc;
     if (row >= rows) return;
     const int cnt = n_pieces[row];
-    const float2 *pl = part_lse + row * c.top_k;
+    const float2 *pl = part_lse + row * slots;
     float mx = -CUDART_INF_F;
     for (int j = 0; j < cnt; ++j) mx = fmaxf(mx, pl[j].x);
     float acc[8];
@@ -571,7 +571,7 @@ tc_merge(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
             den += w;
             const uint32_t eb = (__float_as_uint(pj.y) >> (8 * (sub >> 2))) & 0xffu;
             const float ws = w * __uint_as_float((eb + 1u) << 23);   // weight x 2^(eb - 126)
-            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(part_o + (row * c.top_k + j) * kD + sub * 8));
+            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(part_o + (row * slots + j) * kD + sub * 8));
             const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -595,6 +595,92 @@ tc_merge(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
     *reinterpret_cast<uint4 *>(out + b * c.q_sb + h * c.q_sh + r * c.q_st + sub * 8) = make_uint4(w[0], w[1], w[2], w[3]);
     if (sub == 0)
         lse[((long long)b * c.Hq + h) * c.Lq + r] = den > 0.f ? (mx + log2f(den)) * kLn2 : -CUDART_INF_F;
+}
+
+// Per row, per-span mode (Algorithm 1 with the gate of Section "Combination"): slot j holds the
+// attention over the part of S_t left of the window, slot top_k the attention over the window; A_t
+// merges the two through their log-sum-exp, and O = sum_t alpha_t A_t with alpha = softmax of the
+// selected anchors' search scores.  16 threads per row, 8 columns each.
+__device__ __forceinline__ void load_piece(const __half *part_o, const float2 *pl, long long slot, int sub, float w,
+                                           float (&dst)[8]) {
+    const uint32_t eb = (__float_as_uint(pl->y) >> (8 * (sub >> 2))) & 0xffu;
+    const float ws = w * __uint_as_float((eb + 1u) << 23);   // weight x 2^(eb - 126)
+    const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(part_o + slot * kD + sub * 8));
+    const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&rw[e]));
+        dst[2 * e] = fmaf(ws, f.x, dst[2 * e]);
+        dst[2 * e + 1] = fmaf(ws, f.y, dst[2 * e + 1]);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+tc_merge_gated(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
+               const int32_t *__restrict__ anchor, const float *__restrict__ score, Call c, int slots, int Lc,
+               long long r0, bf16 *__restrict__ out, float *__restrict__ lse, float *__restrict__ lse_span) {
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long row = gid >> 4;
+    const int sub = (int)(gid & 15);
+    const long long rows = (long long)c.B * c.Hq * Lc;
+    if (row >= rows) return;
+    const int rc = (int)(row % Lc);
+    const int bh = (int)(row / Lc);
+    const int h = bh % c.Hq, b = bh / c.Hq;
+    const long long r = r0 + rc, i = c.q_pos0 + r;
+    const long long orow = ((long long)b * c.Hq + h) * c.Lq + r;
+    const int32_t *an = anchor + orow * c.top_k;
+    const float *sc = score + orow * c.top_k;
+    const float2 *pl = part_lse + row * slots;
+    const long long ell = base_len(i, c.span_len);
+    const long long w_lo = i - c.window + 1 > 0 ? i - c.window + 1 : 0;
+    const bool has_w = c.window > 0;
+    const float lw = has_w ? pl[c.top_k].x : -CUDART_INF_F;
+
+    float smax = -CUDART_INF_F;
+    int n_sel = 0;
+    for (int j = 0; j < c.top_k; ++j)
+        if (an[j] >= 0 && an[j] <= i) { smax = fmaxf(smax, sc[j]); ++n_sel; }
+    float sden = 0.f;
+    for (int j = 0; j < c.top_k; ++j)
+        if (an[j] >= 0 && an[j] <= i) sden += expf(sc[j] - smax);
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    float lse_first = -CUDART_INF_F;
+    if (n_sel == 0) {
+        if (has_w) {   // Algorithm 1, empty selection: the window alone
+            load_piece(part_o, pl + c.top_k, row * slots + c.top_k, sub, 1.f, acc);
+            lse_first = lw * kLn2;
+        }
+    }
+    bool first = true;
+    for (int j = 0; j < c.top_k; ++j) {
+        const long long t = an[j];
+        float l_t = -CUDART_INF_F;
+        if (t >= 0 && t <= i) {
+            const long long a = t - (long long)c.back * ell;
+            const bool has_s = !has_w || (a > 0 ? a : 0) < w_lo;   // a part of S_t lies left of the window
+            const float lj = has_s ? pl[j].x : -CUDART_INF_F;
+            const float m = fmaxf(lj, lw);
+            const float wj = has_s ? exp2f(lj - m) : 0.f, ww = has_w ? exp2f(lw - m) : 0.f;
+            const float den = wj + ww;
+            const float alpha = expf(sc[j] - smax) / sden;
+            if (has_s) load_piece(part_o, pl + j, row * slots + j, sub, alpha * wj / den, acc);
+            if (has_w) load_piece(part_o, pl + c.top_k, row * slots + c.top_k, sub, alpha * ww / den, acc);
+            l_t = (m + log2f(den)) * kLn2;
+            if (first) { lse_first = l_t; first = false; }
+        }
+        if (lse_span && sub == 0) lse_span[orow * c.top_k + j] = l_t;
+    }
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 pp = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
+        w[e] = *reinterpret_cast<const uint32_t *>(&pp);
+    }
+    *reinterpret_cast<uint4 *>(out + b * c.q_sb + h * c.q_sh + r * c.q_st + sub * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+    if (sub == 0) lse[orow] = lse_first;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -650,10 +736,10 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 bool tc_attention_shape_ok(const Call &c, int dtype) {
     if (dtype != SLA_BF16 || c.D != kD) return false;
-    if (c.window != 0 || c.mode != SLA_UNION) return false;
     if (c.kv_st < kD || c.top_k > kMaxTopK || !(c.softmax_scale > 0.f)) return false;
     const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
-    const long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
+    long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
+    if (c.window > span_tokens) span_tokens = c.window;
     return span_tokens / kBK + 2 <= 4096;
 }
 
@@ -669,6 +755,7 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     p.NB = (int)((c.Lkv + kBK - 1) / kBK);
     const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
+    if (c.window > span_tokens) span_tokens = c.window;   // the window is a piece too
     if (span_tokens > c.Lkv) span_tokens = c.Lkv;
     p.nb_max = (int)((span_tokens - 1) / kBK + 2);
     // pieces of a group are ordered by blocks covered, in as many classes as the CTA-local histogram
@@ -678,7 +765,8 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     p.ok = (size_t)p.NB * p.ncls * 4 <= 160 * 1024;
     p.ctas_per_bg = (148 + p.n_bg - 1) / p.n_bg;
     const size_t rows = (size_t)c.B * c.Hq * Lc;
-    const size_t slots = rows * c.top_k;
+    p.slots = c.top_k + (c.window > 0 ? 1 : 0);
+    const size_t slots = rows * p.slots;
     const size_t n_keys = (size_t)p.n_bg * p.NB * p.ncls;
     p.max_tiles = (long long)(slots / kRows) + (long long)p.n_bg * p.NB + 1;
     size_t off = 0;
@@ -705,7 +793,7 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         plan = plan_attention_tc(c, (int)Lc);
     }
     if (plan.bytes > scratch_bytes || !plan.ok) return cudaErrorMemoryAllocation;
-    if (plan.max_tiles > (1ll << 30) || (long long)c.B * c.Hq * Lc * c.top_k > (1ll << 31) - 1) return cudaErrorInvalidValue;
+    if (plan.max_tiles > (1ll << 30) || (long long)c.B * c.Hq * Lc * plan.slots > (1ll << 31) - 1) return cudaErrorInvalidValue;
 
     CUtensorMap tm_k, tm_v;
     int slot[3];
@@ -726,6 +814,7 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         tc::PrepArgs pa;
         pa.anchor = anchor; pa.B = c.B; pa.Hq = c.Hq; pa.Hkv = c.Hkv; pa.G = c.G; pa.top_k = c.top_k;
         pa.span_len = c.span_len; pa.back = c.back; pa.fwd = c.fwd; pa.Lq = c.Lq; pa.q_pos0 = c.q_pos0;
+        pa.window = c.window; pa.mode = c.mode;
         pa.r0 = r0; pa.Lc = lc; pa.NB = plan.NB; pa.nb_max = plan.nb_max; pa.ncls = plan.ncls;
         pa.ctas_per_bg = plan.ctas_per_bg;
         pa.key_count = (int *)(ws + plan.off_key_count);
@@ -741,7 +830,7 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         if (e != cudaSuccess) return e;
         TcParams tp;
         tp.q = (const bf16 *)q; tp.q_sb = c.q_sb; tp.q_sh = c.q_sh; tp.q_st = c.q_st;
-        tp.Hq = c.Hq; tp.G = c.G; tp.Lc = lc; tp.top_k = c.top_k; tp.r0 = r0;
+        tp.Hq = c.Hq; tp.G = c.G; tp.Lc = lc; tp.slots = plan.slots; tp.r0 = r0;
         tp.scale2 = c.softmax_scale * kLog2e;
         tp.slot_t = slot[0]; tp.slot_h = slot[1]; tp.slot_b = slot[2];
         tp.recs = pa.recs; tp.tiles = pa.tiles;
@@ -752,7 +841,11 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         tc_attend<<<2 * sm_count, kThreads, kSmemBytes, st>>>(tm_k, tm_v, tp);
         if (timer) timer->end(st);
         const unsigned mblocks = (unsigned)((rows * 16 + 255) / 256);
-        tc_merge<<<mblocks, 256, 0, st>>>(tp.part_o, tp.part_lse, pa.n_pieces, c, lc, r0, (bf16 *)out, lse);
+        if (c.mode == SLA_PER_SPAN)
+            tc_merge_gated<<<mblocks, 256, 0, st>>>(tp.part_o, tp.part_lse, anchor, score, c, plan.slots, lc, r0,
+                                                    (bf16 *)out, lse, lse_span);
+        else
+            tc_merge<<<mblocks, 256, 0, st>>>(tp.part_o, tp.part_lse, pa.n_pieces, c, plan.slots, lc, r0, (bf16 *)out, lse);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         if (launches) *launches += 2;

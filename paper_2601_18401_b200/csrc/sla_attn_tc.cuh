@@ -11,13 +11,14 @@ constexpr int kBK = 64;     // keys per block
 constexpr int kRows = 128;  // pieces per tile
 
 // Work list of one chunk of query positions, as laid out in the scratch memory:
-//   recs   int4 {row, piece index j, lo, hi}: every piece of every row, ordered by
+//   recs   int4 {row, slot of the row's partial results, lo, hi}: every piece of every row, ordered by
 //          (batch*Hkv + kv head, 64-key block of hi, class of blocks covered)
 //   tiles  int4 {batch*Hkv + kv head, end block, first record, records | key blocks to walk << 8}
 //   n_tiles, n_pieces[row], and the per-piece partial results
 struct PrepArgs {
     const int32_t *anchor;   // [B,Hq,Lq,top_k]
     int B, Hq, Hkv, G, top_k, span_len, back, fwd;
+    int window, mode;        // local window w (0 = none); sla_mode_t
     long long Lq, q_pos0, r0;
     int Lc;                  // query positions in this chunk
     int NB;                  // 64-key blocks in [0, Lkv)
@@ -35,18 +36,56 @@ struct PrepArgs {
     int *status;
 };
 
-// Pieces of one row: spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)]),
-// sorted by (lo, hi), clipped so that each key is kept once.  Returns the number of pieces;
-// lo[]/hi[] hold them left to right.
+// Pieces of one row and the slot each one's partial result goes to (slots per row: top_k, plus one
+// when there is a local window W = [max(0, i-w+1), i]).
+//   union mode     the spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)])
+//                  and W, sorted by (lo, hi) and clipped so that each key is kept once; slots are the
+//                  pieces' ordinals left to right;
+//   per-span mode  J_t = S_t united with W is attended as two disjoint pieces: the part of S_t left of
+//                  W in slot j (the anchor's index in the selection) and W, once per row, in slot top_k.
+// Returns the number of pieces; lo[], hi[], slot[] need top_k + 1 entries.
 __device__ inline int row_pieces(const int32_t *__restrict__ an, int top_k, long long i, long long ell,
-                                 int back, int fwd, int *lo, int *hi, int *status) {
+                                 int back, int fwd, int window, int mode, int *lo, int *hi, int *slot,
+                                 int *status) {
+    const int w_lo = (int)(i - window + 1 > 0 ? i - window + 1 : 0);
     int n = 0;
-    for (int j = 0; j < top_k; ++j) {
-        const long long t = an[j];
-        if (t > i) { atomicOr(status, kStatusBadIndex); continue; }
-        if (t < 0) continue;
-        const long long a = t - (long long)back * ell, z = t + (long long)fwd * ell;
-        const int l0 = (int)(a > 0 ? a : 0), h0 = (int)(z < i ? z : i);
+    if (mode == SLA_PER_SPAN) {
+        for (int j = 0; j < top_k; ++j) {
+            const long long t = an[j];
+            if (t > i) { atomicOr(status, kStatusBadIndex); continue; }
+            if (t < 0) continue;
+            const long long a = t - (long long)back * ell, z = t + (long long)fwd * ell;
+            const int l0 = (int)(a > 0 ? a : 0);
+            int h0 = (int)(z < i ? z : i);
+            if (window > 0 && h0 >= w_lo) h0 = w_lo - 1;
+            if (l0 > h0) continue;
+            lo[n] = l0;
+            hi[n] = h0;
+            slot[n] = j;
+            ++n;
+        }
+        if (window > 0) {
+            lo[n] = w_lo;
+            hi[n] = (int)i;
+            slot[n] = top_k;
+            ++n;
+        }
+        return n;
+    }
+    for (int j = 0; j <= top_k; ++j) {
+        int l0, h0;
+        if (j == top_k) {
+            if (window <= 0) break;
+            l0 = w_lo;
+            h0 = (int)i;
+        } else {
+            const long long t = an[j];
+            if (t > i) { atomicOr(status, kStatusBadIndex); continue; }
+            if (t < 0) continue;
+            const long long a = t - (long long)back * ell, z = t + (long long)fwd * ell;
+            l0 = (int)(a > 0 ? a : 0);
+            h0 = (int)(z < i ? z : i);
+        }
         int pos = n;   // insertion sort by (lo, hi)
         while (pos > 0 && (lo[pos - 1] > l0 || (lo[pos - 1] == l0 && hi[pos - 1] > h0))) {
             lo[pos] = lo[pos - 1];
@@ -65,6 +104,7 @@ __device__ inline int row_pieces(const int32_t *__restrict__ an, int top_k, long
         if (j0 <= h0) {
             lo[cnt] = (int)j0;
             hi[cnt] = h0;
+            slot[cnt] = cnt;
             ++cnt;
         }
         if ((long long)h0 + 1 > next_free) next_free = (long long)h0 + 1;

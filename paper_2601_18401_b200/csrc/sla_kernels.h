@@ -31,6 +31,7 @@ cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int
 // Scratch layout for one chunk of Lc query positions (all offsets in bytes).
 struct TcPlan {
     int Lc, n_bg, NB, nb_max, ncls, ctas_per_bg;
+    int slots;   // partial results per query row: top_k, plus one for the local window
     bool ok;   // false when the shared-memory histogram of the counting sort cannot hold NB buckets
     long long max_tiles;
     size_t off_counters, off_key_count, off_key_cursor, off_tiles, off_recs, off_npieces, off_part_lse,

@@ -47,6 +47,8 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
     const int bg = (int)(gid / c.Lq), g = bg % c.Hkv, b = bg / c.Hkv;
     const long long i = c.q_pos0 + r;
     const int n = (int)isqrt_ll(i + 1);
+    // Algorithm 1: anchors inside the local window are no candidates; t_s lies in W iff (s+1)^2 <= w
+    const int s_min = (int)isqrt_ll(c.window);
     float *sc = smem + (size_t)warp * (heads * n_max + 2 * kCap);
     float *cand_v = sc + heads * n_max;
     int *cand_s = reinterpret_cast<int *>(cand_v + kCap);
@@ -65,7 +67,7 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
         }
     }
     const bf16 *kbase = k + b * c.kv_sb + g * c.kv_sh + 8 * q;
-    for (int a0 = 0; a0 < n; a0 += 16) {
+    for (int a0 = s_min; a0 < n; a0 += 16) {
         const int s0 = a0 + r8, s1 = s0 + 8;
         const long long t0 = s0 < n ? i + 1 - (long long)(s0 + 1) * (s0 + 1) : i;
         const long long t1 = s1 < n ? i + 1 - (long long)(s1 + 1) * (s1 + 1) : i;
@@ -83,26 +85,27 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
         }
         // acc[0],acc[1]: anchor s0, heads 2q, 2q+1;  acc[2],acc[3]: anchor s1
         if (2 * q < heads) {
-            if (s0 < n) sc[(2 * q) * n_max + s0] = acc[0] * c.search_scale;
-            if (s1 < n) sc[(2 * q) * n_max + s1] = acc[2] * c.search_scale;
+            if (s0 < n) sc[(2 * q) * n_max + s0 - s_min] = acc[0] * c.search_scale;
+            if (s1 < n) sc[(2 * q) * n_max + s1 - s_min] = acc[2] * c.search_scale;
         }
         if (2 * q + 1 < heads) {
-            if (s0 < n) sc[(2 * q + 1) * n_max + s0] = acc[1] * c.search_scale;
-            if (s1 < n) sc[(2 * q + 1) * n_max + s1] = acc[3] * c.search_scale;
+            if (s0 < n) sc[(2 * q + 1) * n_max + s0 - s_min] = acc[1] * c.search_scale;
+            if (s1 < n) sc[(2 * q + 1) * n_max + s1 - s_min] = acc[3] * c.search_scale;
         }
     }
     __syncwarp();
     for (int hh = 0; hh < heads; ++hh) {
         const int h = g * c.G + head0 + hh;
         const long long obase = ((((long long)b * c.Hq + h) * c.Lq) + r) * c.top_k;
-        select_topk(sc + hh * n_max, n, c.top_k, i, cand_v, cand_s, out_anchor + obase, out_score + obase, lane);
+        select_topk(sc + hh * n_max, n > s_min ? n - s_min : 0, c.top_k, i, cand_v, cand_s, out_anchor + obase,
+                    out_score + obase, lane, s_min);
     }
 }
 
 }  // namespace
 
 bool search_mma_supported(const Call &c, int dtype) {
-    if (dtype != SLA_BF16 || c.D != 128 || c.window != 0) return false;
+    if (dtype != SLA_BF16 || c.D != 128) return false;
     const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
     const int heads = c.G < 8 ? c.G : 8;
     return (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float) <= 200 * 1024;

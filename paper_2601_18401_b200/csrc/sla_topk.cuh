@@ -16,9 +16,11 @@ __device__ __forceinline__ uint32_t order_key(float x) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Top-k of sc[0..n) for one head; writes anchors/scores.  All lanes of the warp take part.
+// Top-k of sc[0..n) for one head, sc[x] being the score of stride index s_base + x (the strides
+// below s_base have their anchors inside the local window and are no candidates); writes
+// anchors/scores.  All lanes of the warp take part.
 __device__ inline void select_topk(float *sc, int n, int top_k, long long i, float *cand_v, int *cand_s,
-                            int32_t *out_anchor, float *out_score, int lane) {
+                            int32_t *out_anchor, float *out_score, int lane, int s_base = 0) {
     const uint32_t kNegInfKey = order_key(-CUDART_INF_F);
     // A. lane maxima over the strided slots
     float lm = -CUDART_INF_F;
@@ -63,7 +65,7 @@ __device__ inline void select_topk(float *sc, int n, int top_k, long long i, flo
                 continue;
             }
             if (bs == smin && order_key(bv) == mx) {
-                out_anchor[j] = (int32_t)(i + 1 - (long long)(bs + 1) * (bs + 1));
+                out_anchor[j] = (int32_t)(i + 1 - (long long)(s_base + bs + 1) * (s_base + bs + 1));
                 out_score[j] = bv;
                 if (first) { v0 = -CUDART_INF_F; s0 = INT_MAX; } else { v1 = -CUDART_INF_F; s1 = INT_MAX; }
             }
@@ -85,7 +87,7 @@ __device__ inline void select_topk(float *sc, int n, int top_k, long long i, flo
             }
             if (lane == 0) {
                 if (bs != INT_MAX) {
-                    out_anchor[j] = (int32_t)(i + 1 - (long long)(bs + 1) * (bs + 1));
+                    out_anchor[j] = (int32_t)(i + 1 - (long long)(s_base + bs + 1) * (s_base + bs + 1));
                     out_score[j] = bv;
                     sc[bs] = -CUDART_INF_F;
                 } else {

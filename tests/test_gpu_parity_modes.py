@@ -86,6 +86,7 @@ def test_chunked_prefill_with_window(sla, handle):
 
 
 def test_single_anchor_modes_agree(sla, handle):
-    """With top_k = 1 the gate is 1 and both modes compute the same attention."""
+    """With top_k = 1 the gate is 1 and both modes compute the same attention (up to the rounding
+    order of the two merge routines: one bf16 step)."""
     r = run_modes(sla, handle, workload(top_k=1, span_len=40), 24)
-    assert torch.equal(r["out"], r["out_g"])
+    assert (r["out"].float() - r["out_g"].float()).abs().max().item() <= 2.0 ** -5
