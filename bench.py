@@ -234,6 +234,45 @@ def max_over_ranks(value: float, dist, device) -> float:
     return float(t.item())
 
 
+def bench_paper_config(sla, handle, dev, steps):
+    """Chunked prefill in the kernel configuration the paper reports (w = 1088, topK = 2, factors 4/2,
+    l(i) = ceil(sqrt(i)), 32K-token chunks), per-span softmax + gate: search and gated attention of
+    every chunk, tokens/s over the whole sequence."""
+    w = synth.CONFIGS[5]
+    x = synth.make_prefill(w, device=dev)
+    B, Hq, L, D = x["q"].shape
+    p = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, window=w.window,
+                        mode=sla.SLA_PER_SPAN, head_dim=D)
+    ch = synth.PAPER_CHUNK
+    anchor = torch.empty(B, Hq, ch, w.top_k, dtype=torch.int32, device=dev)
+    score = torch.empty(B, Hq, ch, w.top_k, dtype=torch.float32, device=dev)
+    lse = torch.empty(B, Hq, ch, dtype=torch.float32, device=dev)
+    lse_span = torch.empty(B, Hq, ch, w.top_k, dtype=torch.float32, device=dev)
+    out = torch.empty_like(x["q"])
+
+    def step():
+        for q0 in range(0, L, ch):
+            qs, q = x["q_s"][:, :, q0:q0 + ch], x["q"][:, :, q0:q0 + ch]
+            sla.sla_span_search(handle, qs, x["k"], p, q_pos0=q0, Lkv=q0 + ch, out_anchor=anchor, out_score=score)
+            sla.sla_span_attention_gated(handle, q, x["k"], x["v"], anchor, score, p, q_pos0=q0, Lkv=q0 + ch,
+                                         out=out[:, :, q0:q0 + ch], lse=lse, lse_span=lse_span)
+
+    for _ in range(3):
+        step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    return {"workload": w.name, "mode": "per-span softmax + gate", "window": w.window, "top_k": w.top_k,
+            "back_factor": w.back_factor, "fwd_factor": w.fwd_factor, "span_len": "ceil(sqrt(i))",
+            "chunk": ch, "ms_per_step": ms, "tokens_per_s": B * L / (ms * 1e-3), "steps": steps}
+
+
 def rank_workload(w, rank: int):
     """Every rank works on its own sequence: same shapes, its own seed (weak scaling, no exchange)."""
     return w.scaled(seed=w.seed + 7919 * rank)
@@ -358,6 +397,8 @@ def run_ours(args, w):
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
     }
 
+    if rank == 0 and not args.no_decode and not args.seq_len:
+        line["paper_kernel_config"] = bench_paper_config(sla, handle, dev, max(3, min(args.steps, 10)))
     if rank == 0 and not args.no_decode:
         del x, anchor, score, out, lse
         torch.cuda.empty_cache()

@@ -93,8 +93,8 @@ typedef struct {
     int32_t back_factor;  /* b >= 0; b >= 2 is needed for full coverage (Section "Span attention") */
     int32_t fwd_factor;   /* f >= 0                                                               */
     int32_t window;       /* local window w of Algorithm 1: W = [max(0,i-w+1), i]; 0 = none;
-                             anchors inside W are no candidates (decode step: only 0)           */
-    int32_t mode;         /* sla_mode_t (decode step: only SLA_UNION)                             */
+                             anchors inside W are no candidates                                  */
+    int32_t mode;         /* sla_mode_t                                                           */
     float search_scale;   /* multiplies the search score (the paper's equation has none: 1.0f)    */
     float softmax_scale;  /* multiplies the attention logits ("scaled dot-product": 1/sqrt(D))     */
 } sla_params_t;
@@ -181,7 +181,10 @@ sla_status_t sla_span_attention_gated(sla_handle_t handle, const void *q, const 
  *   q_s, q     in   [B, Hq, D] device (strides q_stride_b, q_stride_h)
  *   k_cache, v_cache in [B, Hkv, capacity >= n_ctx, D] device (kv strides)
  *   out        out  [B, Hq, D] input dtype, strides as q;  lse out [B, Hq] fp32 contiguous
- *   out_anchor out  [B, Hq, top_k] int32 contiguous; out_score out [B, Hq, top_k] fp32 contiguous  */
+ *   out_anchor out  [B, Hq, top_k] int32 contiguous; out_score out [B, Hq, top_k] fp32 contiguous
+ * params->window and params->mode act as in the prefill calls: anchors inside the window are no
+ * candidates, the window is attended with the spans; in the SLA_PER_SPAN mode `out` is the gated sum
+ * of Algorithm 1 and `lse` the log-sum-exp of the first selected span.                             */
 sla_status_t sla_decode_step(sla_handle_t handle, const void *q_s, const void *q, const void *k_cache,
                              const void *v_cache, int64_t n_ctx, const sla_layout_t *layout,
                              const sla_params_t *params, void *out, float *lse, int32_t *out_anchor,
@@ -202,6 +205,8 @@ sla_status_t sla_decode_step(sla_handle_t handle, const void *q_s, const void *q
  *
  * Arguments, results and launch behaviour are those of sla_decode_step (same kernels); inputs and
  * outputs are still the caller's device buffers.  Differences:
+ *   - only the union mode without a local window (params->window = 0, params->mode = SLA_UNION);
+ *     anything else returns SLA_ERR_UNSUPPORTED;
  *   - a step whose scratch exceeds the fixed array (it grows with batch * heads * sqrt(n_ctx) and
  *     with batch * heads * splits) is rejected with SLA_ERR_WORKSPACE and nothing is launched; the
  *     1M- and 10M-token configurations with 32 query heads need well under 1 MiB;

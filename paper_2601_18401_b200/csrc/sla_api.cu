@@ -62,13 +62,6 @@ const char *check_layout_params(const sla_layout_t *l, const sla_params_t *p, bo
     return nullptr;
 }
 
-// The decode step implements the union mode without a window only.
-sla_status_t check_supported_decode(sla_handle_t h, const sla_params_t *p) {
-    if (p->window != 0) return fail(h, SLA_ERR_UNSUPPORTED, "window > 0 is not implemented for the decode step%s");
-    if (p->mode != SLA_UNION) return fail(h, SLA_ERR_UNSUPPORTED, "only SLA_UNION is implemented for the decode step%s");
-    return SLA_OK;
-}
-
 sla::Call make_call(const sla_handle_t h, const sla_layout_t *l, const sla_params_t *p, int64_t Lq,
                     int64_t q_pos0, int64_t Lkv) {
     sla::Call c;
@@ -311,13 +304,13 @@ sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, con
         return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
     if (!aligned16(q_s) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
         return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
-    if (sla_status_t s = check_supported_decode(h, p)) return s;
     sla::Call c = make_call(h, l, p, 1, n_ctx - 1, n_ctx);
     const sla::DecodePlan plan =
         sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim));
     if (plan.bytes + kHeaderBytes > h->ws_bytes) return fail(h, SLA_ERR_WORKSPACE, "workspace too small for this decode step%s");
     if ((size_t)plan.n_anchor * sizeof(float) * 8 > 180 * 1024) return fail(h, SLA_ERR_UNSUPPORTED, "context too long for the decode top-k stage%s");
-    if ((size_t)(l->batch) * (l->n_kv_heads + l->n_q_heads) * sizeof(int) > kHeaderBytes - kCounterOffset)
+    const size_t units = p->mode == SLA_PER_SPAN ? (size_t)p->top_k : 1;
+    if ((size_t)(l->batch) * (l->n_kv_heads + l->n_q_heads * (units + 1)) * sizeof(int) > kHeaderBytes - kCounterOffset)
         return fail(h, SLA_ERR_UNSUPPORTED, "too many (batch, head) pairs for the decode step%s");
     cudaError_t e = sla::launch_decode(q_s, q, k_cache, v_cache, c, l->dtype, n_ctx, plan, h->ws + kHeaderBytes,
                                        reinterpret_cast<int *>(h->ws + kCounterOffset), out, lse, out_anchor,

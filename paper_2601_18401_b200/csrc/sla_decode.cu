@@ -7,9 +7,12 @@
 //   decode_score   grid (anchor chunks, B*Hkv, head tiles)   K anchor rows x G routing queries; the CTA
 //                  that finishes a (batch, KV head) last selects the k best anchors of its G heads,
 //                  builds their spans and clips the overlaps
-//   decode_attn    grid (n_splits, B*Hq)                     online softmax over an even token share;
-//                  the CTA that finishes a head last merges the split results through their
-//                  log-sum-exp
+//   decode_attn    grid (n_splits, attention units)          online softmax over an even token share;
+//                  the CTA that finishes a unit last merges the split results through their
+//                  log-sum-exp.  Union mode: one unit per head (its spans and the local window, clipped to
+//                  disjoint pieces).  Per-span mode (Algorithm 1 literally): one unit per selected anchor,
+//                  J_t = S_t united with the window; the unit that finishes a head last applies the gate
+//                  of Section "Combination" to the units' outputs
 // "Last" is decided by an atomic counter per (batch, KV head) / per head in the handle's header
 // region; the last CTA puts the counter back to zero, so a step leaves them as it found them.
 #include <limits.h>
@@ -34,7 +37,7 @@ template <int LPR> __device__ inline float reduce_sub(float x) {
 // ------------------------------------------------------------------------------------------------
 template <typename T, int D, int GT>
 __global__ void __launch_bounds__(kScoreThreads)
-decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long long n_ctx, int n,
+decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long long n_ctx, int n, int s_min,
              float *__restrict__ scores, int *__restrict__ done, int *__restrict__ spans,
              int32_t *__restrict__ out_anchor, float *__restrict__ out_score) {
     extern __shared__ float dsm[];
@@ -63,7 +66,8 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
 #pragma unroll
         for (int t = 0; t < GT; ++t) part[u][t] = 0.f;
         if (s < n) {
-            const long long tpos = i + 1 - (long long)(s + 1) * (s + 1);
+            // candidate x is stride s_min + x: the first s_min strides land inside the local window
+            const long long tpos = i + 1 - (long long)(s_min + s + 1) * (s_min + s + 1);
             float kv[E];
             Vec16<T>::load(kbase + tpos * c.kv_st + sub * E, kv);
 #pragma unroll
@@ -95,36 +99,80 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    const int per_warp = n + 2 * topk::kCap + 4 * kMaxTopK;
+    constexpr int kIv = kMaxTopK + 1;   // the spans and the window
+    const int per_warp = n + 2 * topk::kCap + 4 * kIv;
     float *sc = dsm + (size_t)warp * per_warp;
     float *cand_v = sc + n;
     int *cand_s = reinterpret_cast<int *>(cand_v + topk::kCap);
-    int *s_lo = cand_s + topk::kCap, *s_hi = s_lo + kMaxTopK, *p_lo = s_hi + kMaxTopK, *p_hi = p_lo + kMaxTopK;
+    int *s_lo = cand_s + topk::kCap, *s_hi = s_lo + kIv, *p_lo = s_hi + kIv, *p_hi = p_lo + kIv;
     const long long ell = base_len(i, c.span_len);
+    // span table of an attention unit: piece starts [pcap], cumulative token counts [pcap + 1], count
+    const int pcap = c.mode == SLA_PER_SPAN ? 2 : c.top_k + 1, tstride = 2 * pcap + 2;
     for (int hg = warp; hg < c.G; hg += kWarps) {
         const long long bh = (long long)b * c.Hq + g * c.G + hg;
         const float *src = scores + bh * n;
         for (int s = lane; s < n; s += 32) sc[s] = __ldcg(src + s);   // written by other SMs: bypass L1
         __syncwarp();
-        topk::select_topk(sc, n, c.top_k, i, cand_v, cand_s, out_anchor + bh * c.top_k, out_score + bh * c.top_k, lane);
-        // spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)]), sorted by
-        // (lo, hi) and clipped to disjoint pieces with their cumulative token counts
-        for (int j = lane; j < c.top_k; j += 32) {
-            const long long t = out_anchor[bh * c.top_k + j];
+        topk::select_topk(sc, n, c.top_k, i, cand_v, cand_s, out_anchor + bh * c.top_k, out_score + bh * c.top_k, lane,
+                          s_min);
+        __syncwarp();
+        // intervals: the spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)])
+        // and, last, the local window W = [max(0, i-w+1), i]
+        const int n_iv = c.top_k + (c.window > 0 ? 1 : 0);
+        const int w_lo = (int)(i - c.window + 1 > 0 ? i - c.window + 1 : 0);
+        for (int j = lane; j < n_iv; j += 32) {
             int lo = INT_MAX, hi = -1;
-            if (t >= 0) {
-                const long long a = t - (long long)c.back * ell, z = t + (long long)c.fwd * ell;
-                lo = (int)(a > 0 ? a : 0);
-                hi = (int)(z < i ? z : i);
+            if (j == c.top_k) {
+                lo = w_lo;
+                hi = (int)i;
+            } else {
+                const long long t = out_anchor[bh * c.top_k + j];
+                if (t >= 0) {
+                    const long long a = t - (long long)c.back * ell, z = t + (long long)c.fwd * ell;
+                    lo = (int)(a > 0 ? a : 0);
+                    hi = (int)(z < i ? z : i);
+                }
             }
             s_lo[j] = lo;
             s_hi[j] = hi;
         }
         __syncwarp();
-        for (int j = lane; j < c.top_k; j += 32) {
+        if (c.mode == SLA_PER_SPAN) {
+            // one attention unit per selected anchor: the part of S_t left of the window, then the window
+            if (lane == 0) {
+                int n_sel = 0;
+                for (int j = 0; j < c.top_k; ++j) n_sel += s_hi[j] >= 0;
+                for (int j = 0; j < c.top_k; ++j) {
+                    int *start = spans + (bh * c.top_k + j) * tstride;
+                    int *cum = start + pcap;
+                    int cnt = 0, total = 0;
+                    cum[0] = 0;
+                    // a head with nothing selected attends to the window alone: its first unit carries it
+                    const bool sel = s_hi[j] >= 0, lone_w = n_sel == 0 && j == 0 && c.window > 0;
+                    if (sel) {
+                        const int hi_cut = c.window > 0 && s_hi[j] >= w_lo ? w_lo - 1 : s_hi[j];
+                        if (s_lo[j] <= hi_cut) {
+                            start[cnt] = s_lo[j];
+                            total += hi_cut - s_lo[j] + 1;
+                            cum[++cnt] = total;
+                        }
+                    }
+                    if ((sel || lone_w) && c.window > 0) {
+                        start[cnt] = w_lo;
+                        total += (int)i - w_lo + 1;
+                        cum[++cnt] = total;
+                    }
+                    start[2 * pcap + 1] = cnt;
+                }
+            }
+            __syncwarp();
+            continue;
+        }
+        // union mode: sort by (lo, hi), clip to disjoint pieces, cumulative token counts
+        for (int j = lane; j < n_iv; j += 32) {
             const int lo = s_lo[j], hi = s_hi[j];
             int rank = 0;
-            for (int m = 0; m < c.top_k; ++m) {
+            for (int m = 0; m < n_iv; ++m) {
                 const int lm = s_lo[m], hm = s_hi[m];
                 rank += (lm < lo) || (lm == lo && (hm < hi || (hm == hi && m < j)));
             }
@@ -133,12 +181,12 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
         }
         __syncwarp();
         if (lane == 0) {
-            int *start = spans + bh * (2 * c.top_k + 2);
-            int *cum = start + c.top_k;
+            int *start = spans + bh * tstride;
+            int *cum = start + pcap;
             int cnt = 0;
             long long next_free = 0, total = 0;
             cum[0] = 0;
-            for (int a = 0; a < c.top_k; ++a) {
+            for (int a = 0; a < n_iv; ++a) {
                 const int lo = p_lo[a], hi = p_hi[a];
                 if (hi < 0) break;
                 const long long j0 = lo > next_free ? lo : next_free;
@@ -150,7 +198,7 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
                 }
                 if ((long long)hi + 1 > next_free) next_free = (long long)hi + 1;
             }
-            start[2 * c.top_k + 1] = cnt;
+            start[2 * pcap + 1] = cnt;
         }
         __syncwarp();
     }
@@ -161,7 +209,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kAttnThreads)
 decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, Call c,
             const int *__restrict__ spans, float *__restrict__ partial, int *__restrict__ done,
-            T *__restrict__ out, float *__restrict__ lse) {
+            float *__restrict__ unit_out, int *__restrict__ done_head, const int32_t *__restrict__ sel_anchor,
+            const float *__restrict__ sel_score, T *__restrict__ out, float *__restrict__ lse) {
     __shared__ int s_last;
     constexpr int E = Vec16<T>::kElems;
     constexpr int LPR = D / E;
@@ -169,19 +218,22 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
     constexpr int U = 4;
     constexpr int kWarps = kAttnThreads / 32;
     constexpr int kSlots = kWarps * RPI;  // token rows the CTA reads per load step
-    __shared__ int s_start[kMaxTopK], s_cum[kMaxTopK + 1];
+    __shared__ int s_start[kMaxTopK + 1], s_cum[kMaxTopK + 2];
     __shared__ float s_m[kSlots], s_l[kSlots];
     __shared__ float s_acc[kWarps][D];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sub = lane % LPR, rsel = lane / LPR;
-    const long long bh = blockIdx.y;
+    // attention unit: a head (union mode) or one selected anchor of a head (per-span mode)
+    const bool per_span = c.mode == SLA_PER_SPAN;
+    const int units = per_span ? c.top_k : 1, pcap = per_span ? 2 : c.top_k + 1;
+    const long long unit = blockIdx.y, bh = unit / units;
     const int h = (int)(bh % c.Hq), b = (int)(bh / c.Hq), g = h / c.G;
     const int n_splits = gridDim.x, split = blockIdx.x;
 
-    const int *sp = spans + bh * (2 * c.top_k + 2);
-    const int cnt = sp[2 * c.top_k + 1];
+    const int *sp = spans + unit * (2 * pcap + 2);
+    const int cnt = sp[2 * pcap + 1];
     for (int j = tid; j < cnt; j += kAttnThreads) s_start[j] = sp[j];
-    for (int j = tid; j <= cnt; j += kAttnThreads) s_cum[j] = sp[c.top_k + j];
+    for (int j = tid; j <= cnt; j += kAttnThreads) s_cum[j] = sp[pcap + j];
     __syncthreads();
     const long long total = cnt > 0 ? s_cum[cnt] : 0;
     const long long f_begin = total * split / n_splits, f_end = total * (split + 1) / n_splits;
@@ -291,23 +343,24 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
             ll += s_l[w] * sc;
             aa += s_acc[w][tid] * sc;
         }
-        float *dst = partial + (bh * n_splits + split) * (D + 2);
+        float *dst = partial + (unit * n_splits + split) * (D + 2);
         if (tid == 0) { dst[0] = mm; dst[1] = ll; }
         dst[2 + tid] = aa;
     }
-    // ---- the CTA that completes this head merges the split results
+    // ---- the CTA that completes this unit merges the split results
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const int prev = atomicAdd(done + bh, 1);
+        const int prev = atomicAdd(done + unit, 1);
         s_last = prev == n_splits - 1;
-        if (s_last) done[bh] = 0;
+        if (s_last) done[unit] = 0;
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    float o_unit = 0.f, lse_unit = -CUDART_INF_F;
     if (tid < D) {
-        const float *src = partial + bh * n_splits * (D + 2);
+        const float *src = partial + unit * n_splits * (D + 2);
         float mm = -CUDART_INF_F;
         for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, __ldcg(src + s * (D + 2)));
         float ll = 0.f, aa = 0.f;
@@ -317,8 +370,58 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
             ll += __ldcg(src + s * (D + 2) + 1) * sc;
             aa += __ldcg(src + s * (D + 2) + 2 + tid) * sc;
         }
-        out[b * c.q_sb + (long long)h * c.q_sh + tid] = from_float<T>(ll > 0.f ? aa / ll : 0.f);
-        if (tid == 0) lse[bh] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
+        o_unit = ll > 0.f ? aa / ll : 0.f;
+        lse_unit = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
+    }
+    if (!per_span) {
+        if (tid < D) {
+            out[b * c.q_sb + (long long)h * c.q_sh + tid] = from_float<T>(o_unit);
+            if (tid == 0) lse[bh] = lse_unit;
+        }
+        return;
+    }
+    // ---- per-span mode: park A_t and its log-sum-exp; the unit that completes the head applies the gate
+    if (tid < D) {
+        float *dst = unit_out + unit * (D + 2);
+        dst[2 + tid] = o_unit;
+        if (tid == 0) dst[0] = lse_unit;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int prev = atomicAdd(done_head + bh, 1);
+        s_last = prev == units - 1;
+        if (s_last) done_head[bh] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid < D) {
+        const int32_t *an = sel_anchor + bh * c.top_k;
+        const float *sc = sel_score + bh * c.top_k;
+        const float *uo = unit_out + bh * units * (D + 2);
+        float smax = -CUDART_INF_F;
+        int n_sel = 0;
+        for (int j = 0; j < c.top_k; ++j)
+            if (an[j] >= 0) { smax = fmaxf(smax, sc[j]); ++n_sel; }
+        float o = 0.f, l_first = -CUDART_INF_F;
+        if (n_sel == 0) {
+            // Algorithm 1, empty selection: the window alone (carried by the head's first unit)
+            o = __ldcg(uo + 2 + tid);
+            l_first = __ldcg(uo);
+        } else {
+            float sden = 0.f;
+            for (int j = 0; j < c.top_k; ++j)
+                if (an[j] >= 0) sden += expf(sc[j] - smax);
+            bool first = true;
+            for (int j = 0; j < c.top_k; ++j) {
+                if (an[j] < 0) continue;
+                o = fmaf(expf(sc[j] - smax) / sden, __ldcg(uo + j * (D + 2) + 2 + tid), o);
+                if (first) { l_first = __ldcg(uo + j * (D + 2)); first = false; }
+            }
+        }
+        out[b * c.q_sb + (long long)h * c.q_sh + tid] = from_float<T>(o);
+        if (tid == 0) lse[bh] = l_first;
     }
 }
 
@@ -332,13 +435,15 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
     float *scores = (float *)(base + p.off_scores);
     int *spans = (int *)(base + p.off_spans);
     float *partial = (float *)(base + p.off_partial);
-    int *done_bg = counters, *done_bh = counters + c.B * c.Hkv;
-    const int n = p.n_anchor;
+    float *unit_out = (float *)(base + p.off_unit_out);
+    const int units = c.mode == SLA_PER_SPAN ? c.top_k : 1;
+    int *done_bg = counters, *done_unit = counters + c.B * c.Hkv, *done_head = done_unit + c.B * c.Hq * units;
+    const int n = p.n_anchor, s_min = (int)isqrt_ll(c.window);
     const int rows_per_cta = (kScoreThreads / 32) * RPI * 2;
     const int gt = c.G % 8 == 0 ? 8 : c.G % 4 == 0 ? 4 : c.G % 2 == 0 ? 2 : 1;
-    dim3 gs((n + rows_per_cta - 1) / rows_per_cta, c.B * c.Hkv, c.G / gt);
+    dim3 gs(n > 0 ? (n + rows_per_cta - 1) / rows_per_cta : 1, c.B * c.Hkv, c.G / gt);
     const T *qs = (const T *)q_s, *kk = (const T *)k;
-    const size_t smem = (size_t)(kScoreThreads / 32) * (n + 2 * topk::kCap + 4 * kMaxTopK) * sizeof(float);
+    const size_t smem = (size_t)(kScoreThreads / 32) * (n + 2 * topk::kCap + 4 * (kMaxTopK + 1)) * sizeof(float);
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
     cudaError_t e = cudaSuccess;
 #define SLA_LAUNCH_SCORE(GT)                                                                                         \
@@ -346,7 +451,7 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
         auto kern = decode_score<T, D, GT>;                                                                          \
         if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
         if (e == cudaSuccess)                                                                                        \
-            kern<<<gs, kScoreThreads, smem, st>>>(qs, kk, c, n_ctx, n, scores, done_bg, spans, out_anchor, out_score); \
+            kern<<<gs, kScoreThreads, smem, st>>>(qs, kk, c, n_ctx, n, s_min, scores, done_bg, spans, out_anchor, out_score); \
     } while (0)
     switch (gt) {
         case 8: SLA_LAUNCH_SCORE(8); break;
@@ -358,8 +463,9 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
     if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    decode_attn<T, D><<<dim3(p.n_splits, c.B * c.Hq), kAttnThreads, 0, st>>>(
-        (const T *)q, kk, (const T *)v, c, spans, partial, done_bh, (T *)out, lse);
+    decode_attn<T, D><<<dim3(p.n_splits, c.B * c.Hq * units), kAttnThreads, 0, st>>>(
+        (const T *)q, kk, (const T *)v, c, spans, partial, done_unit, unit_out, done_head, out_anchor, out_score,
+        (T *)out, lse);
     return cudaGetLastError();
 }
 
@@ -384,23 +490,29 @@ int decode_attn_blocks_per_sm(int dtype, int D) {
 
 DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots) {
     DecodePlan p;
-    p.n_anchor = (int)isqrt_ll(n_ctx);
+    // candidates: the strides whose anchor lies left of the local window
+    const long long n_cand = isqrt_ll(n_ctx) - isqrt_ll(c.window);
+    p.n_anchor = (int)(n_cand > 0 ? n_cand : 0);
     const long long ell = base_len(n_ctx - 1, c.span_len);
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     if (span_tokens > n_ctx) span_tokens = n_ctx;
-    const long long max_tokens = span_tokens * c.top_k;
-    // one resident wave: as many splits per head as fit the CTA slots of the device
-    long long ns = (long long)cta_slots / ((long long)c.B * c.Hq);
+    const bool per_span = c.mode == SLA_PER_SPAN;
+    const int units = per_span ? c.top_k : 1, pcap = per_span ? 2 : c.top_k + 1;
+    const long long win = c.window < n_ctx ? c.window : n_ctx;
+    const long long max_tokens = per_span ? span_tokens + win : span_tokens * c.top_k + win;
+    // one resident wave: as many splits per attention unit as fit the CTA slots of the device
+    long long ns = (long long)cta_slots / ((long long)c.B * c.Hq * units);
     if (ns > max_tokens / 128) ns = max_tokens / 128;
     if (ns > 256) ns = 256;
     if (ns < 1) ns = 1;
     p.n_splits = (int)ns;
     auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
-    const size_t bh = (size_t)c.B * c.Hq;
+    const size_t bh = (size_t)c.B * c.Hq, n_units = bh * units;
     p.off_scores = 0;
     p.off_spans = align(p.off_scores + bh * (size_t)p.n_anchor * sizeof(float));
-    p.off_partial = align(p.off_spans + bh * (size_t)(2 * c.top_k + 2) * sizeof(int));
-    p.bytes = align(p.off_partial + bh * (size_t)p.n_splits * (c.D + 2) * sizeof(float));
+    p.off_partial = align(p.off_spans + n_units * (size_t)(2 * pcap + 2) * sizeof(int));
+    p.off_unit_out = align(p.off_partial + n_units * (size_t)p.n_splits * (c.D + 2) * sizeof(float));
+    p.bytes = align(p.off_unit_out + (per_span ? n_units * (size_t)(c.D + 2) * sizeof(float) : 0));
     return p;
 }
 

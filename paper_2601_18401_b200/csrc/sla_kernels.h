@@ -49,17 +49,21 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
 // ---- decode step (sla_decode.cu) ---------------------------------------------------------------
 // Scratch layout of one decode step, all offsets in bytes from the scratch base.
 struct DecodePlan {
-    int n_anchor;       // anchors of the query position, floor(sqrt(n_ctx))
-    int n_splits;       // CTAs that share one query head's tokens
+    int n_anchor;       // anchor candidates of the query position: floor(sqrt(n_ctx)) - floor(sqrt(window))
+    int n_splits;       // CTAs that share one attention unit's tokens (unit: a head, or one selected
+                        // anchor of a head in the per-span mode)
     size_t off_scores;  // float [B*Hq][n_anchor]
-    size_t off_spans;   // int   [B*Hq][2*top_k + 2]: piece start, cumulative token offset, total, count
-    size_t off_partial; // float [B*Hq][n_splits][D + 2]: running max, denominator, numerator
+    size_t off_spans;   // int   [units][2*P + 2]: piece starts, cumulative token counts, piece count
+                        //       (P = top_k + 1 in the union mode, 2 in the per-span mode)
+    size_t off_partial; // float [units][n_splits][D + 2]: running max, denominator, numerator
+    size_t off_unit_out; // float [units][D + 2] (per-span mode): log-sum-exp and output of every unit
     size_t bytes;
 };
 // cta_slots = SM count x resident decode_attn CTAs per SM (see decode_attn_blocks_per_sm)
 DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots);
 int decode_attn_blocks_per_sm(int dtype, int D);
-// counters: B*Hkv + B*Hq ints, zero on entry and zero again on exit (completion counters)
+// counters: B*Hkv + B*Hq*units + B*Hq ints (units = top_k in the per-span mode, else 1), zero on entry
+// and zero again on exit (completion counters)
 cudaError_t launch_decode(const void *q_s, const void *q, const void *k, const void *v, const Call &c,
                           int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, int *counters,
                           void *out, float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st);

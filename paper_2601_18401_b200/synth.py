@@ -44,14 +44,20 @@ class Workload:
         return replace(self, **kw)
 
 
-# The five benchmark configurations (index 0..4).
+# The five benchmark configurations (index 0..4) and, last, the kernel configuration the paper reports
+# its throughput with (Section "Experimental setup", "Kernel configuration": w = 1088, topK = 2,
+# backward/forward factors 4 and 2, l(i) = ceil(sqrt(i)), 32K-token prefill chunks) on the shapes of
+# the second configuration.
 CONFIGS = [
     Workload("tiny_prefill_L4096", "prefill", 1, 1, 1, 64, 4096, "f32", 64, 4, seed=1001),
     Workload("prefill_L65536", "prefill", 1, 32, 8, 128, 65536, "bf16", 256, 8, planted_spans=16, seed=1002),
     Workload("prefill_stress_L262144", "prefill", 2, 16, 4, 128, 262144, "bf16", 512, 16, seed=1003),
     Workload("decode_1M", "decode", 1, 32, 4, 128, 1048576, "bf16", 1024, 16, steps=256, seed=1004),
     Workload("decode_10M", "decode", 1, 32, 4, 128, 10485760, "bf16", 3072, 16, steps=128, seed=1005),
+    Workload("prefill_paper_kernel_config_L65536", "prefill", 1, 32, 8, 128, 65536, "bf16", 0, 2, back_factor=4,
+             fwd_factor=2, window=1088, seed=1006),
 ]
+PAPER_CHUNK = 32768   # query positions per call in the paper's chunked prefill
 
 
 def torch_dtype(name: str) -> torch.dtype:

@@ -90,3 +90,44 @@ def test_single_anchor_modes_agree(sla, handle):
     order of the two merge routines: one bf16 step)."""
     r = run_modes(sla, handle, workload(top_k=1, span_len=40), 24)
     assert (r["out"].float() - r["out_g"].float()).abs().max().item() <= 2.0 ** -5
+
+
+@pytest.mark.parametrize("mode", ["union", "per_span"])
+@pytest.mark.parametrize("window,n_ctx0,span_len,top_k,dtype,D,Hq,Hkv", [
+    (0, 3000, 40, 4, "bf16", 128, 8, 2),
+    (64, 3000, 40, 4, "bf16", 128, 8, 2),
+    (1088, 5000, 0, 2, "bf16", 128, 4, 4),       # the paper's window; l(i) = ceil(sqrt(i))
+    (100, 700, 16, 5, "f32", 64, 3, 1),
+    (900, 800, 16, 3, "bf16", 128, 4, 2),        # window covers the whole context: nothing to select
+])
+def test_decode_modes_and_window(sla, handle, mode, window, n_ctx0, span_len, top_k, dtype, D, Hq, Hkv):
+    """Decode step with the local window and in both modes against the oracle's decode step."""
+    from paper_2601_18401_b200 import synth
+    w = synth.Workload("dm", "decode", 2, Hq, Hkv, D, n_ctx0, dtype, span_len, top_k, seed=91)
+    steps = 3
+    kc, vc = synth.make_decode_cache(w, "cuda:0", capacity=n_ctx0 + steps)
+    hk, hv = synth.to_numpy(kc), synth.to_numpy(vc)
+    code = synth.dtype_code(dtype)
+    m_gpu = sla.SLA_PER_SPAN if mode == "per_span" else sla.SLA_UNION
+    m_ref = O.PER_SPAN if mode == "per_span" else O.UNION
+    params = sla.make_params(top_k, span_len, window=window, mode=m_gpu, head_dim=D)
+    for s in range(steps):
+        x = synth.make_decode_step_inputs(w, s, "cuda:0")
+        n_ctx = n_ctx0 + s + 1
+        kc[:, :, n_ctx - 1] = x["k_new"]
+        vc[:, :, n_ctx - 1] = x["v_new"]
+        hk[:, :, n_ctx - 1] = synth.to_numpy(x["k_new"])
+        hv[:, :, n_ctx - 1] = synth.to_numpy(x["v_new"])
+        out, lse, anchor, score = sla.sla_decode_step(handle, x["q_s"], x["q"], kc, vc, n_ctx, params)
+        torch.cuda.synchronize()
+        assert sla.sla_poll_status(handle) == sla.SLA_OK
+        ref = O.decode_step(synth.to_numpy(x["q_s"]), synth.to_numpy(x["q"]), hk, hv, code, n_ctx=n_ctx,
+                            top_k=top_k, span_len=span_len, window=window, mode=m_ref)
+        rs = {k_: ref[k_][:, :, None] for k_ in ("anchor", "score", "gap")}
+        P.compare_search(anchor[:, :, None], score[:, :, None], rs, q_pos0=n_ctx - 1)
+        # attention parity on the GPU's own anchors and scores
+        att = O.span_attention(synth.to_numpy(x["q"])[:, :, None], hk, hv, code,
+                               anchor.cpu().numpy()[:, :, None], span_len=span_len, window=window, mode=m_ref,
+                               score=score.cpu().numpy().astype(np.float64)[:, :, None],
+                               q_pos0=n_ctx - 1, Lkv=n_ctx)
+        P.compare_attention(out[:, :, None], lse[:, :, None], att, dtype)
