@@ -557,22 +557,38 @@ tc_merge(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
     if (row >= rows) return;
     const int cnt = n_pieces[row];
     const float2 *pl = part_lse + row * slots;
-    float mx = -CUDART_INF_F;
-    for (int j = 0; j < cnt; ++j) mx = fmaxf(mx, pl[j].x);
+    const __half *po = part_o + row * slots * kD + sub * 8;
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    float den = 0.f;
-    if (mx > -CUDART_INF_F) {
-        for (int j = 0; j < cnt; ++j) {
-            const float2 pj = pl[j];
-            if (pj.x == -CUDART_INF_F) continue;
-            const float w = exp2f(pj.x - mx);
+    // running maximum and denominator (log2 domain); the pieces come four at a time so that their
+    // loads are in flight together
+    float mx = -CUDART_INF_F, den = 0.f;
+    for (int j0 = 0; j0 < cnt; j0 += 4) {
+        float2 pj[4];
+        uint4 raw[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const bool on = j0 + u < cnt;
+            pj[u] = on ? __ldg(pl + j0 + u) : make_float2(-CUDART_INF_F, 0.f);
+            raw[u] = on ? __ldg(reinterpret_cast<const uint4 *>(po + (long long)(j0 + u) * kD)) : make_uint4(0, 0, 0, 0);
+        }
+        float bm = fmaxf(fmaxf(pj[0].x, pj[1].x), fmaxf(pj[2].x, pj[3].x));
+        if (bm > mx) {
+            const float r = mx == -CUDART_INF_F ? 0.f : exp2f(mx - bm);
+            den *= r;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] *= r;
+            mx = bm;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (pj[u].x == -CUDART_INF_F) continue;
+            const float w = exp2f(pj[u].x - mx);
             den += w;
-            const uint32_t eb = (__float_as_uint(pj.y) >> (8 * (sub >> 2))) & 0xffu;
+            const uint32_t eb = (__float_as_uint(pj[u].y) >> (8 * (sub >> 2))) & 0xffu;
             const float ws = w * __uint_as_float((eb + 1u) << 23);   // weight x 2^(eb - 126)
-            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(part_o + (row * slots + j) * kD + sub * 8));
-            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+            const uint32_t rw[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&rw[e]));
