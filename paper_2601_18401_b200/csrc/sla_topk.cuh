@@ -51,24 +51,28 @@ __device__ inline void select_topk(float *sc, int n, int top_k, long long i, flo
     }
     __syncwarp();
     if (count <= kCap) {
-        // D. k rounds of warp arg-max over the candidates (two per lane)
-        float v0 = lane < count ? cand_v[lane] : -CUDART_INF_F, v1 = lane + 32 < count ? cand_v[lane + 32] : -CUDART_INF_F;
-        int s0 = lane < count ? cand_s[lane] : INT_MAX, s1 = lane + 32 < count ? cand_s[lane + 32] : INT_MAX;
-        for (int j = 0; j < top_k; ++j) {
-            const bool first = v0 > v1 || (v0 == v1 && s0 <= s1);
-            const float bv = first ? v0 : v1;
-            const int bs = first ? s0 : s1;
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, order_key(bv));
-            const int smin = __reduce_min_sync(0xffffffffu, (order_key(bv) == mx && bs != INT_MAX) ? bs : INT_MAX);
-            if (smin == INT_MAX) {   // fewer candidates than slots: pad
-                if (lane == 0) { out_anchor[j] = -1; out_score[j] = -CUDART_INF_F; }
-                continue;
+        // D. rank of every candidate among the candidates (larger score first, smaller stride index on
+        // ties: a strict total order on the order keys); ranks below top_k are the output slots
+        uint32_t *cand_k = reinterpret_cast<uint32_t *>(cand_v);
+        for (int cidx = lane; cidx < count; cidx += 32) cand_k[cidx] = order_key(cand_v[cidx]);
+        __syncwarp();
+        for (int cidx = lane; cidx < count; cidx += 32) {
+            const uint32_t kc = cand_k[cidx];
+            const int sc_ = cand_s[cidx];
+            int rank = 0;
+            for (int x = 0; x < count; ++x) {
+                const uint32_t kx = cand_k[x];
+                rank += (kx > kc) || (kx == kc && cand_s[x] < sc_);
             }
-            if (bs == smin && order_key(bv) == mx) {
-                out_anchor[j] = (int32_t)(i + 1 - (long long)(s_base + bs + 1) * (s_base + bs + 1));
-                out_score[j] = bv;
-                if (first) { v0 = -CUDART_INF_F; s0 = INT_MAX; } else { v1 = -CUDART_INF_F; s1 = INT_MAX; }
+            if (rank < top_k) {
+                const long long m = s_base + sc_ + 1;
+                out_anchor[rank] = (int32_t)(i + 1 - m * m);
+                out_score[rank] = __uint_as_float((kc & 0x80000000u) ? (kc & 0x7fffffffu) : ~kc);
             }
+        }
+        for (int j = count + lane; j < top_k; j += 32) {   // fewer candidates than slots: pad
+            out_anchor[j] = -1;
+            out_score[j] = -CUDART_INF_F;
         }
     } else {
         // many equal scores at the threshold: plain k rounds over all scores
