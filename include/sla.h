@@ -227,7 +227,11 @@ sla_status_t sla_decode_step_static(const void *q_s, const void *q, const void *
 
 /* sla_span_search followed by sla_span_attention on HOST buffers (pinned memory gives the best
  * copy rate): copies q_s, q, k, v to the device, runs both steps, copies out, lse, anchors and
- * scores back, and waits for completion.  All tensors are dense and contiguous
+ * scores back, and waits for completion.  Sequences of 8192 tokens and more go through in up to
+ * eight chunks of query positions (chunked prefill: a chunk needs the keys up to its own end), with
+ * the copy-in of the next chunk, the kernels of this one and the copy-out of the previous one
+ * overlapping on streams the handle owns; results do not depend on the chunking.  Union mode only.
+ * All tensors are dense and contiguous
  * ([B,Hq,L,D] / [B,Hkv,L,D], q_pos0 = 0, Lq = Lkv = L); the layout's strides are ignored.  The
  * device staging buffers come out of the handle's workspace, which therefore has to be
  * sla_workspace_bytes(...) + sla_host_staging_bytes(...) large.  Section references as above. */

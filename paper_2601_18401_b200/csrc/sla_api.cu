@@ -17,6 +17,10 @@ struct sla_handle_s {
     size_t scratch_avail = 0; // bytes of workspace after the header that kernels may use as scratch
     sla::KernelTimer timer;   // sla_set_kernel_timing / sla_kernel_time_ms
     bool force_simt = false;  // environment SLA_FORCE_SIMT=1: generic kernels only (for A/B checks)
+    // sla_prefill_host: copy-in and copy-out streams and per-chunk events, created on first use
+    static constexpr int kMaxChunks = 16;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_in[kMaxChunks] = {}, ev_done[kMaxChunks] = {};
     char err[256] = {0};
 };
 
@@ -185,6 +189,14 @@ sla_status_t sla_destroy(sla_handle_t h) {
     if (!h) return SLA_ERR_INVALID_ARG;
     for (int j = 0; j < 2 * sla::KernelTimer::kMaxPairs; ++j)
         if (h->timer.ev[j]) cudaEventDestroy(h->timer.ev[j]);
+    for (int j = 0; j < sla_handle_s::kMaxChunks; ++j) {
+        if (h->ev_in[j]) cudaEventDestroy(h->ev_in[j]);
+        if (h->ev_done[j]) cudaEventDestroy(h->ev_done[j]);
+    }
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->s_in) cudaStreamDestroy(h->s_in);
+    if (h->s_out) cudaStreamDestroy(h->s_out);
     cudaError_t e = cudaFree(h->ws);
     delete h;
     return e == cudaSuccess ? SLA_OK : SLA_ERR_CUDA;
@@ -359,22 +371,78 @@ sla_status_t sla_prefill_host(sla_handle_t h, const void *q_s_host, const void *
     float *d_lse = (float *)take(rows * 4);
     int32_t *d_anchor = (int32_t *)take(rows * p->top_k * 4);
     float *d_score = (float *)take(rows * p->top_k * 4);
-    cudaError_t e = cudaMemcpyAsync(d_qs, q_s_host, qb, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(d_k, k_host, kb, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(d_q, q_host, qb, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(d_v, v_host, kb, cudaMemcpyHostToDevice, st);
+
+    // The sequence goes through in chunks of query positions (chunked prefill: chunk c needs the keys
+    // up to its own end only), so that the copy-in of chunk c+1, the kernels of chunk c and the
+    // copy-out of chunk c-1 overlap on three streams.  The device tensors keep the host layout
+    // [B, H, L, D]; a chunk of positions is a 2-D copy (one segment per (batch, head)).  Anchors, scores
+    // and lse of a chunk are compact [B, Hq, Lc, ...] blocks, as the search call writes them.
+    int n_chunks = (int)(L / 4096);
+    if (n_chunks > 8) n_chunks = 8;
+    if (n_chunks < 1) n_chunks = 1;
+    const int64_t Lc = ((L + n_chunks - 1) / n_chunks + 127) / 128 * 128;
+    n_chunks = (int)((L + Lc - 1) / Lc);
+    cudaError_t e = cudaSuccess;
+    if (!h->s_in) {
+        e = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+        for (int j = 0; j < sla_handle_s::kMaxChunks && e == cudaSuccess; ++j) {
+            e = cudaEventCreateWithFlags(&h->ev_in[j], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_done[j], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) return cuda_fail(h, e, "sla_prefill_host (streams)");
+    }
+    const size_t D = (size_t)l->head_dim;
+    const size_t row_q = (size_t)L * D * es;          // pitch of one (batch, head) segment
+    const int nq = l->batch * l->n_q_heads, nkv = l->batch * l->n_kv_heads;
+    // copy-in stream: ordered after whatever the caller's stream holds so far
+    e = cudaEventRecord(h->ev_fork, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->s_in, h->ev_fork, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->s_out, h->ev_fork, 0);
+    for (int c = 0; c < n_chunks && e == cudaSuccess; ++c) {
+        const int64_t c0 = (int64_t)c * Lc, lc = (L - c0 < Lc) ? L - c0 : Lc;
+        const size_t off = (size_t)c0 * D * es, width = (size_t)lc * D * es;
+        e = cudaMemcpy2DAsync(d_qs + off, row_q, (const char *)q_s_host + off, row_q, width, nq, cudaMemcpyHostToDevice, h->s_in);
+        if (e == cudaSuccess) e = cudaMemcpy2DAsync(d_k + off, row_q, (const char *)k_host + off, row_q, width, nkv, cudaMemcpyHostToDevice, h->s_in);
+        if (e == cudaSuccess) e = cudaMemcpy2DAsync(d_q + off, row_q, (const char *)q_host + off, row_q, width, nq, cudaMemcpyHostToDevice, h->s_in);
+        if (e == cudaSuccess) e = cudaMemcpy2DAsync(d_v + off, row_q, (const char *)v_host + off, row_q, width, nkv, cudaMemcpyHostToDevice, h->s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(h->ev_in[c], h->s_in);
+    }
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_prefill_host (copy in)");
     const size_t avail_before = h->scratch_avail;
     h->scratch_avail = h->ws_bytes - kHeaderBytes - stage;   // the staging buffers are not scratch
-    sla_status_t s = sla_span_search(h, d_qs, d_k, L, 0, L, &dl, p, d_anchor, d_score, stream);
-    if (s == SLA_OK) s = sla_span_attention(h, d_q, d_k, d_v, L, 0, L, &dl, p, d_anchor, d_out, d_lse, stream);
+    sla_status_t s = SLA_OK;
+    const size_t k4 = (size_t)p->top_k * 4;
+    for (int c = 0; c < n_chunks && s == SLA_OK; ++c) {
+        const int64_t c0 = (int64_t)c * Lc, lc = (L - c0 < Lc) ? L - c0 : Lc;
+        const size_t off = (size_t)c0 * D * es;
+        // compact per-chunk blocks: chunk c starts after the rows of the chunks before it
+        const size_t blk = (size_t)nq * c0;
+        int32_t *a_c = d_anchor + blk * p->top_k;
+        float *s_c = d_score + blk * p->top_k, *l_c = d_lse + blk;
+        e = cudaStreamWaitEvent(st, h->ev_in[c], 0);
+        if (e != cudaSuccess) { s = cuda_fail(h, e, "sla_prefill_host (wait)"); break; }
+        s = sla_span_search(h, d_qs + off, d_k, lc, c0, c0 + lc, &dl, p, a_c, s_c, stream);
+        if (s == SLA_OK) s = sla_span_attention(h, d_q + off, d_k, d_v, lc, c0, c0 + lc, &dl, p, a_c, d_out + off, l_c, stream);
+        if (s != SLA_OK) break;
+        e = cudaEventRecord(h->ev_done[c], st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->s_out, h->ev_done[c], 0);
+        const size_t width = (size_t)lc * D * es;
+        if (e == cudaSuccess) e = cudaMemcpy2DAsync((char *)out_host + off, row_q, d_out + off, row_q, width, nq, cudaMemcpyDeviceToHost, h->s_out);
+        if (e == cudaSuccess) e = cudaMemcpy2DAsync((char *)lse_host + (size_t)c0 * 4, (size_t)L * 4, l_c, (size_t)lc * 4, (size_t)lc * 4, nq, cudaMemcpyDeviceToHost, h->s_out);
+        if (e == cudaSuccess) e = cudaMemcpy2DAsync((char *)anchor_host + (size_t)c0 * k4, (size_t)L * k4, a_c, (size_t)lc * k4, (size_t)lc * k4, nq, cudaMemcpyDeviceToHost, h->s_out);
+        if (e == cudaSuccess) e = cudaMemcpy2DAsync((char *)score_host + (size_t)c0 * k4, (size_t)L * k4, s_c, (size_t)lc * k4, (size_t)lc * k4, nq, cudaMemcpyDeviceToHost, h->s_out);
+        if (e != cudaSuccess) s = cuda_fail(h, e, "sla_prefill_host (copy out)");
+    }
     h->scratch_avail = avail_before;
-    if (s != SLA_OK) return s;
-    e = cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(lse_host, d_lse, rows * 4, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(anchor_host, d_anchor, rows * p->top_k * 4, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(score_host, d_score, rows * p->top_k * 4, cudaMemcpyDeviceToHost, st);
+    // join: the caller's stream continues after the last copy-out, and this call returns after it
+    e = cudaEventRecord(h->ev_join, h->s_out);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, h->ev_join, 0);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->s_in);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (s != SLA_OK) return s;
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_prefill_host (copy out)");
     return SLA_OK;
 }

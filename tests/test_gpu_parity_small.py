@@ -177,3 +177,37 @@ def test_error_returns(sla, handle):
         sla.sla_decode_step(small, qq, qq, kc, kc, 100000, sla.make_params(4, 16))
     assert e.value.status == -3
     small.close()
+
+
+@pytest.mark.parametrize("seq_len,dtype", [(9000, "bf16"), (12345, "bf16"), (8300, "f32"), (700, "bf16")])
+def test_prefill_host_matches_device_calls(sla, seq_len, dtype):
+    """sla_prefill_host (chunked, copies overlapped with the kernels) against the two device calls on
+    the whole sequence and against the oracle: same anchors, outputs within the parity bounds."""
+    from paper_2601_18401_b200 import synth
+    w = workload(seq_len=seq_len, dtype=dtype, span_len=24, top_k=5, n_q_heads=4, n_kv_heads=2,
+                 head_dim=128 if dtype == "bf16" else 64)
+    x = synth.make_prefill(w, device="cuda:0")
+    params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
+    layout = sla.make_layout(x["q"], x["k"])
+    handle = sla.Handle(0, sla.sla_workspace_bytes(layout, params, seq_len, seq_len)
+                        + sla.sla_host_staging_bytes(layout, params, seq_len) + (16 << 20))
+    anchor, score = sla.sla_span_search(handle, x["q_s"], x["k"], params)
+    out, lse = sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params)
+    host = {n: t.cpu().pin_memory() for n, t in x.items()}
+    for rep in range(2):   # the second call reuses the handle's streams and events
+        ho, hl, ha, hs = sla.sla_prefill_host(handle, host["q_s"], host["q"], host["k"], host["v"], params)
+        assert sla.sla_poll_status(handle) == sla.SLA_OK
+        assert torch.equal(ha, anchor.cpu()) and torch.equal(hs, score.cpu())
+        tol = P.OUT_TOL[dtype]
+        assert (ho.float() - out.cpu().float()).abs().max().item() <= tol
+        fin = torch.isfinite(lse.cpu())
+        assert torch.equal(torch.isfinite(hl), fin)
+        assert (hl[fin] - lse.cpu()[fin]).abs().max().item() <= P.LSE_TOL[dtype]
+    rows = np.unique(np.concatenate([np.arange(0, 40), np.arange(seq_len - 40, seq_len),
+                                     np.random.default_rng(5).integers(0, seq_len, 200)]))
+    hn = P.host_inputs(x)
+    code = synth.dtype_code(dtype)
+    ref = O.span_attention(hn["q"], hn["k"], hn["v"], code, np.ascontiguousarray(ha[:, :, rows].numpy()),
+                           span_len=w.span_len, rows=rows)
+    P.compare_attention(ho, hl, ref, dtype, rows=rows)
+    handle.close()
