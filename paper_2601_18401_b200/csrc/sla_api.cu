@@ -378,7 +378,7 @@ sla_status_t sla_prefill_host(sla_handle_t h, const void *q_s_host, const void *
     // [B, H, L, D]; a chunk of positions is a 2-D copy (one segment per (batch, head)).  Anchors, scores
     // and lse of a chunk are compact [B, Hq, Lc, ...] blocks, as the search call writes them.
     int n_chunks = (int)(L / 4096);
-    if (n_chunks > 8) n_chunks = 8;
+    if (n_chunks > sla_handle_s::kMaxChunks) n_chunks = sla_handle_s::kMaxChunks;
     if (n_chunks < 1) n_chunks = 1;
     const int64_t Lc = ((L + n_chunks - 1) / n_chunks + 127) / 128 * 128;
     n_chunks = (int)((L + Lc - 1) / Lc);
