@@ -41,10 +41,10 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
            float *__restrict__ out_score, int n_max, int head0, int heads) {
     extern __shared__ float smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long gid = (long long)blockIdx.x * kWarps + warp;   // (b, g, r)
-    if (gid >= (long long)c.B * c.Hkv * c.Lq) return;
-    const long long r = gid % c.Lq;
-    const int bg = (int)(gid / c.Lq), g = bg % c.Hkv, b = bg / c.Hkv;
+    // grid: x = groups of kWarps query positions, y = batch * Hkv + kv head (no 64-bit divisions here)
+    const long long r = (long long)blockIdx.x * kWarps + warp;
+    if (r >= c.Lq) return;
+    const int bg = blockIdx.y, g = bg % c.Hkv, b = bg / c.Hkv;
     const long long i = c.q_pos0 + r;
     const int n = (int)isqrt_ll(i + 1);
     // Algorithm 1: anchors inside the local window are no candidates; t_s lies in W iff (s+1)^2 <= w
@@ -67,15 +67,17 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
         }
     }
     const bf16 *kbase = k + b * c.kv_sb + g * c.kv_sh + 8 * q;
+    const int kv_st = (int)c.kv_st, i32 = (int)i;   // positions and the token stride fit 31 bits: 32x32->64 products
     for (int a0 = s_min; a0 < n; a0 += 16) {
         const int s0 = a0 + r8, s1 = s0 + 8;
-        const long long t0 = s0 < n ? i + 1 - (long long)(s0 + 1) * (s0 + 1) : i;
-        const long long t1 = s1 < n ? i + 1 - (long long)(s1 + 1) * (s1 + 1) : i;
+        const int t0 = s0 < n ? i32 + 1 - (s0 + 1) * (s0 + 1) : i32;
+        const int t1 = s1 < n ? i32 + 1 - (s1 + 1) * (s1 + 1) : i32;
+        const bf16 *row0 = kbase + (long long)t0 * kv_st, *row1 = kbase + (long long)t1 * kv_st;
         uint4 ra[4], rb[4];
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
-            ra[ch] = __ldg(reinterpret_cast<const uint4 *>(kbase + t0 * c.kv_st + 32 * ch));
-            rb[ch] = __ldg(reinterpret_cast<const uint4 *>(kbase + t1 * c.kv_st + 32 * ch));
+            ra[ch] = __ldg(reinterpret_cast<const uint4 *>(row0 + 32 * ch));
+            rb[ch] = __ldg(reinterpret_cast<const uint4 *>(row1 + 32 * ch));
         }
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -105,7 +107,7 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
 }  // namespace
 
 bool search_mma_supported(const Call &c, int dtype) {
-    if (dtype != SLA_BF16 || c.D != 128) return false;
+    if (dtype != SLA_BF16 || c.D != 128 || (long long)c.B * c.Hkv > 65535 || c.kv_st > INT_MAX) return false;
     const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
     const int heads = c.G < 8 ? c.G : 8;
     return (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float) <= 200 * 1024;
@@ -114,8 +116,7 @@ bool search_mma_supported(const Call &c, int dtype) {
 cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int32_t *oa, float *os, cudaStream_t st,
                               long long *launches) {
     const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
-    const long long groups = (long long)c.B * c.Hkv * c.Lq;
-    const unsigned blocks = (unsigned)((groups + kWarps - 1) / kWarps);
+    const dim3 blocks((unsigned)((c.Lq + kWarps - 1) / kWarps), (unsigned)(c.B * c.Hkv));
     for (int head0 = 0; head0 < c.G; head0 += 8) {
         const int heads = c.G - head0 < 8 ? c.G - head0 : 8;
         const size_t smem = (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float);
