@@ -149,7 +149,12 @@ def run_reference(args, w):
         return
     x = synth.make_prefill(w, device="cpu")
     host = {n: synth.to_numpy(t) for n, t in x.items()}
-    rows = oracle_sample_rows(w.seq_len, args.ref_rows)
+    # the sample of one step is bounded so that the whole run stays near 150 s of oracle time: a
+    # calibration pass on 256 positions gives the rate, the per-step sample follows from it
+    calib = oracle_sample_rows(w.seq_len, 256)
+    rate = len(calib) / time_oracle_prefill(w, host, calib)
+    n_rows = int(min(args.ref_rows, max(64, 150.0 * rate / max(1, args.steps))))
+    rows = oracle_sample_rows(w.seq_len, n_rows)
     for _ in range(args.warmup):
         time_oracle_prefill(w, host, rows[: max(4, len(rows) // 16)])
     secs = [time_oracle_prefill(w, host, rows) for _ in range(args.steps)]

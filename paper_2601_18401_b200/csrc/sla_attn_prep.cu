@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
     int lo[kMaxTopK + 1], hi[kMaxTopK + 1], slot[kMaxTopK + 1];
     // sub-pass A: this CTA's pieces per bucket
     for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
-        const int hg = (int)(q / a.Lc), rc = (int)(q % a.Lc);
+        const int hg = (int)((unsigned)q / (unsigned)a.Lc), rc = (int)((unsigned)q % (unsigned)a.Lc);   // G * Lc < 2^31
         const int h = g * a.G + hg;
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
         const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
     __syncthreads();
     // sub-pass B: write the records
     for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
-        const int hg = (int)(q / a.Lc), rc = (int)(q % a.Lc);
+        const int hg = (int)((unsigned)q / (unsigned)a.Lc), rc = (int)((unsigned)q % (unsigned)a.Lc);   // G * Lc < 2^31
         const int h = g * a.G + hg;
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
         const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;

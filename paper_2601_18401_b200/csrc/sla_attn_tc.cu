@@ -598,8 +598,8 @@ tc_merge(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
         }
     }
     const float inv = den > 0.f ? 1.f / den : 0.f;
-    const int rc = (int)(row % Lc);
-    const int bh = (int)(row / Lc);
+    const int rc = (int)((unsigned)row % (unsigned)Lc);   // rows < 2^31
+    const int bh = (int)((unsigned)row / (unsigned)Lc);
     const int h = bh % c.Hq, b = bh / c.Hq;
     const long long r = r0 + rc;
     uint32_t w[4];
@@ -640,8 +640,8 @@ tc_merge_gated(const __half *__restrict__ part_o, const float2 *__restrict__ par
     const int sub = (int)(gid & 15);
     const long long rows = (long long)c.B * c.Hq * Lc;
     if (row >= rows) return;
-    const int rc = (int)(row % Lc);
-    const int bh = (int)(row / Lc);
+    const int rc = (int)((unsigned)row % (unsigned)Lc);   // rows < 2^31
+    const int bh = (int)((unsigned)row / (unsigned)Lc);
     const int h = bh % c.Hq, b = bh / c.Hq;
     const long long r = r0 + rc, i = c.q_pos0 + r;
     const long long orow = ((long long)b * c.Hq + h) * c.Lq + r;
