@@ -663,32 +663,59 @@ tc_merge_gated(const __half *__restrict__ part_o, const float2 *__restrict__ par
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    float lse_first = -CUDART_INF_F;
-    if (n_sel == 0) {
-        if (has_w) {   // Algorithm 1, empty selection: the window alone
-            load_piece(part_o, pl + c.top_k, row * slots + c.top_k, sub, 1.f, acc);
-            lse_first = lw * kLn2;
-        }
+    // O = sum_t alpha_t (w_t o_t + ww_t o_W) / den_t: the window piece enters once, with the summed
+    // coefficient cw; the spans' pieces come four at a time so that their loads are in flight together
+    float lse_first = -CUDART_INF_F, cw = 0.f;
+    if (n_sel == 0 && has_w) {   // Algorithm 1, empty selection: the window alone
+        cw = 1.f;
+        lse_first = lw * kLn2;
     }
     bool first = true;
-    for (int j = 0; j < c.top_k; ++j) {
-        const long long t = an[j];
-        float l_t = -CUDART_INF_F;
-        if (t >= 0 && t <= i) {
+    const __half *po = part_o + row * slots * kD + sub * 8;
+    for (int j0 = 0; j0 < c.top_k; j0 += 4) {
+        float2 pj[4];
+        uint4 raw[4];
+        bool sel[4], has_s[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u;
+            const long long t = j < c.top_k ? an[j] : -1;
+            sel[u] = t >= 0 && t <= i;
             const long long a = t - (long long)c.back * ell;
-            const bool has_s = !has_w || (a > 0 ? a : 0) < w_lo;   // a part of S_t lies left of the window
-            const float lj = has_s ? pl[j].x : -CUDART_INF_F;
-            const float m = fmaxf(lj, lw);
-            const float wj = has_s ? exp2f(lj - m) : 0.f, ww = has_w ? exp2f(lw - m) : 0.f;
-            const float den = wj + ww;
-            const float alpha = expf(sc[j] - smax) / sden;
-            if (has_s) load_piece(part_o, pl + j, row * slots + j, sub, alpha * wj / den, acc);
-            if (has_w) load_piece(part_o, pl + c.top_k, row * slots + c.top_k, sub, alpha * ww / den, acc);
-            l_t = (m + log2f(den)) * kLn2;
-            if (first) { lse_first = l_t; first = false; }
+            has_s[u] = sel[u] && (!has_w || (a > 0 ? a : 0) < w_lo);   // a part of S_t lies left of the window
+            pj[u] = has_s[u] ? __ldg(pl + j) : make_float2(-CUDART_INF_F, 0.f);
+            raw[u] = has_s[u] ? __ldg(reinterpret_cast<const uint4 *>(po + (long long)j * kD)) : make_uint4(0, 0, 0, 0);
         }
-        if (lse_span && sub == 0) lse_span[orow * c.top_k + j] = l_t;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u;
+            if (j >= c.top_k) break;
+            float l_t = -CUDART_INF_F;
+            if (sel[u]) {
+                const float lj = pj[u].x;
+                const float m = fmaxf(lj, lw);
+                const float wj = has_s[u] ? exp2f(lj - m) : 0.f, ww = has_w ? exp2f(lw - m) : 0.f;
+                const float den = wj + ww;
+                const float alpha = expf(sc[j] - smax) / sden;
+                cw = fmaf(alpha, ww / den, cw);
+                if (has_s[u]) {
+                    const uint32_t eb = (__float_as_uint(pj[u].y) >> (8 * (sub >> 2))) & 0xffu;
+                    const float ws = alpha * wj / den * __uint_as_float((eb + 1u) << 23);   // weight x 2^(eb - 126)
+                    const uint32_t rw[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&rw[e]));
+                        acc[2 * e] = fmaf(ws, f.x, acc[2 * e]);
+                        acc[2 * e + 1] = fmaf(ws, f.y, acc[2 * e + 1]);
+                    }
+                }
+                l_t = (m + log2f(den)) * kLn2;
+                if (first) { lse_first = l_t; first = false; }
+            }
+            if (lse_span && sub == 0) lse_span[orow * c.top_k + j] = l_t;
+        }
     }
+    if (cw != 0.f) load_piece(part_o, pl + c.top_k, row * slots + c.top_k, sub, cw, acc);
     uint32_t w[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
