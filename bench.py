@@ -38,7 +38,9 @@ METRIC = "prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one tc_attend launch of the default workload
 # (L = 65536), from the one-pass ncu capture of the full-size launch summarised in profiles/
-TC_ATTEND_DRAM_BYTES_PER_LAUNCH = {65536: 7.52e9, 16384: 1.43e9}
+TC_ATTEND_DRAM_BYTES_PER_LAUNCH = {65536: 7.37e9, 16384: 1.43e9}
+# the same for one decode_attn launch (the dominant kernel of a decode step), by workload
+DECODE_ATTN_DRAM_BYTES_PER_LAUNCH = {"decode_1M": 487.6e6, "decode_10M": 1572.6e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -227,7 +229,7 @@ def bench_decode(sla, handle, w, steps, peaks, dev):
             "algorithmic_bytes_per_step": bytes_step,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0,
-                         "traffic": None, "peak_source": peaks["_source"]}}
+                         "traffic": DECODE_ATTN_DRAM_BYTES_PER_LAUNCH.get(w.name), "peak_source": peaks["_source"]}}
 
 
 def max_over_ranks(value: float, dist, device) -> float:
