@@ -30,7 +30,8 @@
  *   - no positional encoding and no padding mask are applied.
  *
  * Memory: unless a parameter says "host", every tensor pointer is DEVICE memory owned by the
- * caller, on the device the handle was created for.  The innermost (head_dim) axis is contiguous;
+ * caller, on the device the handle was created for, which must be the CURRENT device of the calling
+ * thread (SLA_ERR_INVALID_ARG otherwise).  The innermost (head_dim) axis is contiguous;
  * the other strides are given in ELEMENTS.  Base pointers must be 16-byte aligned and every stride
  * a multiple of 8 elements.  Calls are asynchronous: work is enqueued on the given CUDA stream
  * (a cudaStream_t passed as void*; NULL = the default stream) and outputs are valid once the stream

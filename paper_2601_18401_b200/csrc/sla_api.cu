@@ -66,6 +66,13 @@ const char *check_layout_params(const sla_layout_t *l, const sla_params_t *p, bo
     return nullptr;
 }
 
+// Kernels are launched on the current device: it has to be the one the handle was created on.
+const char *check_device(const sla_handle_t h) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != h->device) return "the handle's device is not the current device";
+    return nullptr;
+}
+
 sla::Call make_call(const sla_handle_t h, const sla_layout_t *l, const sla_params_t *p, int64_t Lq,
                     int64_t q_pos0, int64_t Lkv) {
     sla::Call c;
@@ -236,6 +243,7 @@ sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int
     if (const char *why = check_layout_params(l, p, false)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (const char *why = check_prefill_range(Lq, q_pos0, Lkv)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!q_s || !k || !out_anchor || !out_score) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!aligned16(q_s) || !aligned16(k)) return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -259,6 +267,7 @@ sla_status_t span_attention_impl(sla_handle_t h, const void *q, const void *k, c
                                  float *lse_span, void *stream, const char *what) {
     if (const char *why = check_prefill_range(Lq, q_pos0, Lkv)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!q || !k || !v || !anchor || !out || !lse) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
         return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
@@ -312,6 +321,7 @@ sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, con
     if (!h) return SLA_ERR_INVALID_ARG;
     if (const char *why = check_layout_params(l, p, true)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (n_ctx <= 0 || n_ctx > 2147483647LL) return fail(h, SLA_ERR_INVALID_ARG, "n_ctx must be in 1..2^31-1%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!q_s || !q || !k_cache || !v_cache || !out || !lse || !out_anchor || !out_score)
         return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
     if (!aligned16(q_s) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
@@ -351,6 +361,7 @@ sla_status_t sla_prefill_host(sla_handle_t h, const void *q_s_host, const void *
     if (L <= 0 || L > 2147483647LL) return fail(h, SLA_ERR_INVALID_ARG, "L out of range%s");
     if (!q_s_host || !q_host || !k_host || !v_host || !out_host || !lse_host || !anchor_host || !score_host)
         return fail(h, SLA_ERR_INVALID_ARG, "NULL host pointer%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     sla_layout_t dl = *l;
     dl.q_stride_t = dl.kv_stride_t = l->head_dim;
     dl.q_stride_h = dl.kv_stride_h = L * l->head_dim;

@@ -203,12 +203,16 @@ __global__ void __launch_bounds__(256) prep_tile_bounds(PrepArgs a) {
 cudaError_t prepare(const PrepArgs &a, cudaStream_t st, long long *launches) {
     const int n_bg = a.B * a.Hkv;
     const size_t smem = (size_t)a.NB * a.ncls * sizeof(int);
-    static size_t attr_bytes = 0;
-    if (smem > 48 * 1024 && smem > attr_bytes) {
+    // function attributes belong to a device's context: remember the largest size set per device
+    static size_t attr_bytes[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    const bool known = dev >= 0 && dev < 64;
+    if (smem > 48 * 1024 && (!known || smem > attr_bytes[dev])) {
         cudaError_t e = cudaFuncSetAttribute(prep_pieces<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(prep_pieces<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_bytes = smem;
+        if (known) attr_bytes[dev] = smem;
     }
     const unsigned grid = (unsigned)(n_bg * a.ctas_per_bg);
     prep_pieces<0><<<grid, kPrepThreads, smem, st>>>(a);

@@ -841,11 +841,14 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
     CUtensorMap tm_k, tm_v;
     int slot[3];
     if (!make_kv_map(&tm_k, k, c, slot) || !make_kv_map(&tm_v, v, c, slot)) return cudaErrorInvalidValue;
-    static bool attr_set = false;
-    if (!attr_set) {
+    // function attributes belong to a device's context: remember them per device, not per process
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(tc_attend, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     char *ws = (char *)scratch;
     int *counters = (int *)(ws + plan.off_counters);
