@@ -87,9 +87,40 @@ int64_t sla_oracle_ceil_isqrt(int64_t x) {
     return r;
 }
 
-/* Base span length l(i): the fixed value when span_len > 0, else the paper's rule. */
-int64_t sla_oracle_base_len(int64_t i, int64_t span_len) {
-    return span_len > 0 ? span_len : sla_oracle_ceil_isqrt(i);
+/*
+ * General exponents (Section "Span attention": anchors at i - (s+1)^(1/p) + 1 for general p; Section
+ * "Training": search_exponent for the stride pattern, span_exponent for the span length).  The paper
+ * does not say how the real number (s+1)^(1/p) becomes a position; reading R18: it is rounded UP to
+ * an integer, after taking off one part in 1e12 so that a power that is an integer in exact
+ * arithmetic (p = 1/3: cubes) is not pushed to the next one by the rounding of 1/p and pow (their
+ * relative error is a few 1e-15; positions stay below 2^31, so the margin is far below 1).  For
+ * p = 1/2 the offsets are the exact squares, computed in integers.
+ */
+static int64_t ceil_pow(double base, double expo) {
+    double x = pow(base, expo);
+    return (int64_t)ceil(x - 1e-12 * x);
+}
+
+/* Distance of the stride-s anchor from position i + 1: o_s = ceil((s+1)^(1/p)). */
+int64_t sla_oracle_stride_offset(int64_t s, double p) {
+    if (p == 0.5) return (s + 1) * (s + 1);
+    return ceil_pow((double)(s + 1), 1.0 / p);
+}
+
+/* Number of strides whose anchor exists for query position i: o_s <= i + 1 (reading R1). */
+int64_t sla_oracle_n_strides(int64_t i, double p) {
+    int64_t n = 0;
+    while (sla_oracle_stride_offset(n, p) <= i + 1) n++;
+    return n;
+}
+
+/* Base span length l(i): the fixed value when span_len > 0, else the paper's rule ceil(i^p_span)
+ * (an exact integer ceil-sqrt for p_span = 1/2). */
+int64_t sla_oracle_base_len(int64_t i, int64_t span_len, double p_span) {
+    if (span_len > 0) return span_len;
+    if (i <= 0) return 0;
+    if (p_span == 0.5) return sla_oracle_ceil_isqrt(i);
+    return ceil_pow((double)i, p_span);
 }
 
 /*
@@ -97,11 +128,11 @@ int64_t sla_oracle_base_len(int64_t i, int64_t span_len) {
  * Writes the key positions in stride order (s ascending, i.e. nearest first) and, when s_out is not
  * NULL, the stride index of each.  Returns how many there are; writes at most cap of them.
  */
-int64_t sla_oracle_anchors(int64_t i, int64_t window, int64_t *t_out, int64_t *s_out, int64_t cap) {
+int64_t sla_oracle_anchors(int64_t i, int64_t window, double p, int64_t *t_out, int64_t *s_out, int64_t cap) {
     int64_t n = 0;
     int64_t w_lo = window > 0 ? (i - window + 1 > 0 ? i - window + 1 : 0) : i + 1; /* W = [w_lo, i] */
     for (int64_t s = 0;; s++) {
-        int64_t t = i - (s + 1) * (s + 1) + 1;
+        int64_t t = i - sla_oracle_stride_offset(s, p) + 1;
         if (t < 0) break;                      /* reading R1 */
         if (window > 0 && t >= w_lo) continue; /* anchor lies inside W: not a candidate */
         if (n < cap) {
@@ -165,11 +196,12 @@ int sla_oracle_threads(void) {
  */
 int sla_oracle_span_search(const void *q_s, const void *k, int dtype, int B, int Hq, int Hkv, int D,
                            int64_t Lq, int64_t q_pos0, int64_t Lkv, int64_t kv_cap, int top_k,
-                           int64_t window, double search_scale, const int64_t *rows, int64_t n_rows,
-                           int32_t *out_anchor, double *out_score, double *out_gap,
-                           int64_t *n_dots) {
+                           int64_t window, double search_scale, double search_exponent,
+                           const int64_t *rows, int64_t n_rows, int32_t *out_anchor, double *out_score,
+                           double *out_gap, int64_t *n_dots) {
     if (!q_s || !k || B <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv || D <= 0 || Lq <= 0 || top_k <= 0 ||
-        q_pos0 < 0 || q_pos0 + Lq > Lkv || Lkv > kv_cap || window < 0)
+        q_pos0 < 0 || q_pos0 + Lq > Lkv || Lkv > kv_cap || window < 0 || !(search_exponent > 0.0) ||
+        !(search_exponent < 1.0))
         return -1;
     const int G = Hq / Hkv;
     const int64_t R = rows ? n_rows : Lq;
@@ -183,11 +215,12 @@ int sla_oracle_span_search(const void *q_s, const void *k, int dtype, int B, int
             const int64_t r = rows ? rows[rr] : rr;
             if (r < 0 || r >= Lq) { bad = 1; continue; }
             const int64_t i = q_pos0 + r;
-            const int64_t n_all = isqrt_fast(i + 1); /* strides with t >= 0 */
+            const int64_t n_all = search_exponent == 0.5 ? isqrt_fast(i + 1)
+                                                         : sla_oracle_n_strides(i, search_exponent); /* strides with t >= 0 */
             double *sc = (double *)malloc(sizeof(double) * (size_t)(n_all > 0 ? n_all : 1));
             int64_t *tt = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n_all > 0 ? n_all : 1));
             char *taken = (char *)calloc((size_t)(n_all > 0 ? n_all : 1), 1);
-            const int64_t n = sla_oracle_anchors(i, window, tt, NULL, n_all);
+            const int64_t n = sla_oracle_anchors(i, window, search_exponent, tt, NULL, n_all);
             const int64_t q_off = (((int64_t)b * Hq + h) * Lq + r) * D;
             for (int64_t c = 0; c < n; c++) {
                 const int64_t k_off = (((int64_t)b * Hkv + g) * kv_cap + tt[c]) * D;
@@ -295,7 +328,7 @@ int sla_oracle_span_attention(const void *q, const void *k, const void *v, int d
                               int Hkv, int D, int64_t Lq, int64_t q_pos0, int64_t Lkv,
                               int64_t kv_cap, int top_k, int64_t span_len, int64_t back_factor,
                               int64_t fwd_factor, int64_t window, int mode, double softmax_scale,
-                              const int64_t *rows, int64_t n_rows, const int32_t *anchor,
+                              double span_exponent, const int64_t *rows, int64_t n_rows, const int32_t *anchor,
                               const double *score, double *out, double *lse, double *lse_span,
                               int64_t *n_pairs) {
     if (!q || !k || !v || !anchor || B <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv || D <= 0 || Lq <= 0 ||
@@ -314,7 +347,7 @@ int sla_oracle_span_attention(const void *q, const void *k, const void *v, int d
             const int64_t r = rows ? rows[rr] : rr;
             if (r < 0 || r >= Lq) { bad = 1; continue; }
             const int64_t i = q_pos0 + r;
-            const int64_t ell = sla_oracle_base_len(i, span_len);
+            const int64_t ell = sla_oracle_base_len(i, span_len, span_exponent);
             const int64_t q_off = (((int64_t)b * Hq + h) * Lq + r) * D;
             const int64_t kv_off = ((int64_t)b * Hkv + g) * kv_cap * D;
             const int64_t row = ((int64_t)b * Hq + h) * R + rr;
@@ -394,15 +427,16 @@ int sla_oracle_decode_step(const void *q_s, const void *q, const void *k_cache, 
                            int dtype, int B, int Hq, int Hkv, int D, int64_t n_ctx, int64_t kv_cap,
                            int top_k, int64_t span_len, int64_t back_factor, int64_t fwd_factor,
                            int64_t window, int mode, double search_scale, double softmax_scale,
+                           double search_exponent, double span_exponent,
                            int32_t *out_anchor, double *out_score, double *out_gap, double *out,
                            double *lse, int64_t *n_dots, int64_t *n_pairs) {
     if (n_ctx <= 0) return -1;
     int rc = sla_oracle_span_search(q_s, k_cache, dtype, B, Hq, Hkv, D, 1, n_ctx - 1, n_ctx, kv_cap,
-                                    top_k, window, search_scale, NULL, 0, out_anchor, out_score,
-                                    out_gap, n_dots);
+                                    top_k, window, search_scale, search_exponent, NULL, 0, out_anchor,
+                                    out_score, out_gap, n_dots);
     if (rc) return rc;
     return sla_oracle_span_attention(q, k_cache, v_cache, dtype, B, Hq, Hkv, D, 1, n_ctx - 1, n_ctx,
                                      kv_cap, top_k, span_len, back_factor, fwd_factor, window, mode,
-                                     softmax_scale, NULL, 0, out_anchor, out_score, out, lse, NULL,
-                                     n_pairs);
+                                     softmax_scale, span_exponent, NULL, 0, out_anchor, out_score, out, lse,
+                                     NULL, n_pairs);
 }

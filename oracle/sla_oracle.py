@@ -44,24 +44,28 @@ def lib():
         _lib.sla_oracle_ceil_isqrt.restype = i64
         _lib.sla_oracle_ceil_isqrt.argtypes = [i64]
         _lib.sla_oracle_base_len.restype = i64
-        _lib.sla_oracle_base_len.argtypes = [i64, i64]
+        _lib.sla_oracle_base_len.argtypes = [i64, i64, dbl]
+        _lib.sla_oracle_stride_offset.restype = i64
+        _lib.sla_oracle_stride_offset.argtypes = [i64, dbl]
+        _lib.sla_oracle_n_strides.restype = i64
+        _lib.sla_oracle_n_strides.argtypes = [i64, dbl]
         _lib.sla_oracle_anchors.restype = i64
-        _lib.sla_oracle_anchors.argtypes = [i64, i64, vp, vp, i64]
+        _lib.sla_oracle_anchors.argtypes = [i64, i64, dbl, vp, vp, i64]
         _lib.sla_oracle_span.restype = None
         _lib.sla_oracle_span.argtypes = [i64, i64, i64, i64, i64, vp, vp]
         _lib.sla_oracle_threads.restype = i32
         _lib.sla_oracle_span_search.restype = i32
         _lib.sla_oracle_span_search.argtypes = (
-            [vp, vp, i32, i32, i32, i32, i32, i64, i64, i64, i64, i32, i64, dbl, vp, i64, vp, vp, vp, vp]
+            [vp, vp, i32, i32, i32, i32, i32, i64, i64, i64, i64, i32, i64, dbl, dbl, vp, i64, vp, vp, vp, vp]
         )
         _lib.sla_oracle_span_attention.restype = i32
         _lib.sla_oracle_span_attention.argtypes = (
-            [vp, vp, vp, i32, i32, i32, i32, i32, i64, i64, i64, i64, i32, i64, i64, i64, i64, i32, dbl,
+            [vp, vp, vp, i32, i32, i32, i32, i32, i64, i64, i64, i64, i32, i64, i64, i64, i64, i32, dbl, dbl,
              vp, i64, vp, vp, vp, vp, vp, vp]
         )
         _lib.sla_oracle_decode_step.restype = i32
         _lib.sla_oracle_decode_step.argtypes = (
-            [vp, vp, vp, vp, i32, i32, i32, i32, i32, i64, i64, i32, i64, i64, i64, i64, i32, dbl, dbl,
+            [vp, vp, vp, vp, i32, i32, i32, i32, i32, i64, i64, i32, i64, i64, i64, i64, i32, dbl, dbl, dbl, dbl,
              vp, vp, vp, vp, vp, vp, vp]
         )
     return _lib
@@ -80,16 +84,26 @@ def ceil_isqrt(x: int) -> int:
     return int(lib().sla_oracle_ceil_isqrt(int(x)))
 
 
-def base_len(i: int, span_len: int = 0) -> int:
-    return int(lib().sla_oracle_base_len(int(i), int(span_len)))
+def base_len(i: int, span_len: int = 0, span_exponent: float = 0.5) -> int:
+    return int(lib().sla_oracle_base_len(int(i), int(span_len), float(span_exponent)))
 
 
-def anchors(i: int, window: int = 0):
+def stride_offset(s: int, search_exponent: float = 0.5) -> int:
+    """Distance of the stride-s anchor from position i + 1."""
+    return int(lib().sla_oracle_stride_offset(int(s), float(search_exponent)))
+
+
+def n_strides(i: int, search_exponent: float = 0.5) -> int:
+    return int(lib().sla_oracle_n_strides(int(i), float(search_exponent)))
+
+
+def anchors(i: int, window: int = 0, search_exponent: float = 0.5):
     """Candidate anchor positions of query ``i`` and their stride indices, nearest first."""
-    n = int(lib().sla_oracle_anchors(int(i), int(window), None, None, 0))
+    p = float(search_exponent)
+    n = int(lib().sla_oracle_anchors(int(i), int(window), p, None, None, 0))
     t = np.zeros(max(n, 1), dtype=np.int64)
     s = np.zeros(max(n, 1), dtype=np.int64)
-    lib().sla_oracle_anchors(int(i), int(window), t.ctypes.data, s.ctypes.data, n)
+    lib().sla_oracle_anchors(int(i), int(window), p, t.ctypes.data, s.ctypes.data, n)
     return t[:n], s[:n]
 
 
@@ -117,7 +131,8 @@ def _rows(rows):
     return r, int(r.size), r.ctypes.data
 
 
-def span_search(q_s, k, dtype, *, top_k, q_pos0=0, Lkv=None, window=0, search_scale=1.0, rows=None):
+def span_search(q_s, k, dtype, *, top_k, q_pos0=0, Lkv=None, window=0, search_scale=1.0, rows=None,
+                search_exponent=0.5):
     """q_s [B,Hq,Lq,D], k [B,Hkv,cap,D] -> dict(anchor, score, gap, n_dots); see the C header comment."""
     q_s, k = _as_input(q_s, dtype), _as_input(k, dtype)
     B, Hq, Lq, D = q_s.shape
@@ -131,7 +146,7 @@ def span_search(q_s, k, dtype, *, top_k, q_pos0=0, Lkv=None, window=0, search_sc
     n_dots = C.c_int64(0)
     rc = lib().sla_oracle_span_search(
         q_s.ctypes.data, k.ctypes.data, dtype, B, Hq, Hkv, D, Lq, int(q_pos0), Lkv, cap, int(top_k),
-        int(window), float(search_scale), rptr, n_rows, anchor.ctypes.data, score.ctypes.data,
+        int(window), float(search_scale), float(search_exponent), rptr, n_rows, anchor.ctypes.data, score.ctypes.data,
         gap.ctypes.data, C.addressof(n_dots))
     if rc:
         raise ValueError("sla_oracle_span_search rejected its arguments")
@@ -139,7 +154,8 @@ def span_search(q_s, k, dtype, *, top_k, q_pos0=0, Lkv=None, window=0, search_sc
 
 
 def span_attention(q, k, v, dtype, anchor, *, span_len, back_factor=2, fwd_factor=0, window=0,
-                   mode=UNION, softmax_scale=None, q_pos0=0, Lkv=None, rows=None, score=None):
+                   mode=UNION, softmax_scale=None, q_pos0=0, Lkv=None, rows=None, score=None,
+                   span_exponent=0.5):
     """q [B,Hq,Lq,D], k/v [B,Hkv,cap,D], anchor [B,Hq,R,k] -> dict(out, lse, lse_span, n_pairs)."""
     q, k, v = _as_input(q, dtype), _as_input(k, dtype), _as_input(v, dtype)
     B, Hq, Lq, D = q.shape
@@ -162,7 +178,7 @@ def span_attention(q, k, v, dtype, anchor, *, span_len, back_factor=2, fwd_facto
     rc = lib().sla_oracle_span_attention(
         q.ctypes.data, k.ctypes.data, v.ctypes.data, dtype, B, Hq, Hkv, D, Lq, int(q_pos0), Lkv, cap,
         int(top_k), int(span_len), int(back_factor), int(fwd_factor), int(window), int(mode),
-        float(softmax_scale), rptr, n_rows, anchor.ctypes.data,
+        float(softmax_scale), float(span_exponent), rptr, n_rows, anchor.ctypes.data,
         None if score is None else score.ctypes.data, out.ctypes.data, lse.ctypes.data,
         lse_span.ctypes.data, C.addressof(n_pairs))
     if rc:
@@ -171,7 +187,8 @@ def span_attention(q, k, v, dtype, anchor, *, span_len, back_factor=2, fwd_facto
 
 
 def decode_step(q_s, q, k_cache, v_cache, dtype, *, n_ctx, top_k, span_len, back_factor=2,
-                fwd_factor=0, window=0, mode=UNION, search_scale=1.0, softmax_scale=None):
+                fwd_factor=0, window=0, mode=UNION, search_scale=1.0, softmax_scale=None,
+                search_exponent=0.5, span_exponent=0.5):
     """q_s,q [B,Hq,D]; caches [B,Hkv,cap,D] -> dict(out, lse, anchor, score, gap, n_dots, n_pairs)."""
     q_s, q = _as_input(q_s, dtype), _as_input(q, dtype)
     k_cache, v_cache = _as_input(k_cache, dtype), _as_input(v_cache, dtype)
@@ -188,7 +205,8 @@ def decode_step(q_s, q, k_cache, v_cache, dtype, *, n_ctx, top_k, span_len, back
     rc = lib().sla_oracle_decode_step(
         q_s.ctypes.data, q.ctypes.data, k_cache.ctypes.data, v_cache.ctypes.data, dtype, B, Hq, Hkv, D,
         int(n_ctx), cap, int(top_k), int(span_len), int(back_factor), int(fwd_factor), int(window),
-        int(mode), float(search_scale), float(softmax_scale), anchor.ctypes.data, score.ctypes.data,
+        int(mode), float(search_scale), float(softmax_scale), float(search_exponent), float(span_exponent),
+        anchor.ctypes.data, score.ctypes.data,
         gap.ctypes.data, out.ctypes.data, lse.ctypes.data, C.addressof(n_dots), C.addressof(n_pairs))
     if rc:
         raise ValueError("sla_oracle_decode_step rejected its arguments")

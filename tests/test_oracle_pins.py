@@ -401,3 +401,92 @@ def test_input_dtypes_are_widened_exactly():
         oa = O.span_attention(as_np[1], as_np[2], as_np[3], code, a["anchor"], span_len=4)
         ob = O.span_attention(as_64[1], as_64[2], as_64[3], O.F64, b["anchor"], span_len=4)
         assert np.array_equal(oa["out"], ob["out"])
+
+
+# ---- general exponents (Section "Span attention": anchors at i - (s+1)^(1/p) + 1; Section "Training":
+# search_exponent / span_exponent, e.g. 1/3 and 2/3) ------------------------------------------------
+
+def icbrt(x: int) -> int:
+    r = round(x ** (1.0 / 3.0))
+    while r ** 3 > x:
+        r -= 1
+    while (r + 1) ** 3 <= x:
+        r += 1
+    return r
+
+
+def test_stride_offsets_for_rational_exponents_are_exact_powers():
+    """p = 1/2, 1/3, 1/4: (s+1)^(1/p) is an integer in exact arithmetic and must come out as that
+    integer (the rounding of 1/p and of pow must not push it to the next one)."""
+    for s in list(range(0, 300)) + [999, 1289]:          # offsets up to 2^31, the largest position
+        assert O.stride_offset(s, 0.5) == (s + 1) ** 2
+        assert O.stride_offset(s, 1.0 / 3.0) == (s + 1) ** 3
+        if (s + 1) ** 4 < 2 ** 31:
+            assert O.stride_offset(s, 0.25) == (s + 1) ** 4
+    for p in (0.5, 1.0 / 3.0, 0.54, 0.4, 0.7):
+        offs = [O.stride_offset(s, p) for s in range(400)]
+        assert offs[0] == 1                                    # stride 0 is the query's own position
+        assert all(b > a for a, b in zip(offs, offs[1:]))      # strictly increasing: distinct anchors
+        # rounded up: the anchor never lies right of the real-valued position i - x + 1
+        assert all(o >= (s + 1) ** (1.0 / p) * (1 - 2e-12) for s, o in enumerate(offs))
+        assert all(o < (s + 1) ** (1.0 / p) + 1 for s, o in enumerate(offs))
+
+
+def test_number_of_strides_matches_integer_roots_and_scales_as_i_to_p():
+    for i in list(range(0, 2000)) + [10 ** 6, 10 ** 9 + 7]:
+        assert O.n_strides(i, 0.5) == math.isqrt(i + 1)
+        assert O.n_strides(i, 1.0 / 3.0) == icbrt(i + 1)
+    for p in (0.4, 0.54, 0.6):
+        n1, n2 = O.n_strides(10 ** 5, p), O.n_strides(10 ** 7, p)
+        assert abs(n1 / (10 ** 5) ** p - 1) < 0.02 and abs(n2 / (10 ** 7) ** p - 1) < 0.01
+        assert abs(math.log(n2 / n1) / math.log(100) - p) < 0.005   # O(i^p) candidates
+
+
+def test_anchors_with_exponent_one_third():
+    t, s = O.anchors(1000, 0, 1.0 / 3.0)
+    assert list(t) == [1001 - m ** 3 for m in range(1, 11)] and list(s) == list(range(10))
+    t, s = O.anchors(1000, 30, 1.0 / 3.0)          # W = [971, 1000]: offsets 1, 8, 27 fall inside
+    assert list(t) == [1001 - m ** 3 for m in range(4, 11)] and list(s) == list(range(3, 10))
+
+
+def test_base_len_with_span_exponent():
+    for k in range(1, 60):
+        assert O.base_len(k ** 3, 0, 2.0 / 3.0) == k * k          # exact at perfect cubes
+        assert O.base_len(k ** 3 + 1, 0, 2.0 / 3.0) == k * k + 1  # rounded up right after
+    assert O.base_len(0, 0, 2.0 / 3.0) == 0 and O.base_len(5, 7, 2.0 / 3.0) == 7
+    for i in (1, 2, 30, 31, 1000, 65535):
+        assert O.base_len(i, 0, 0.5) == math.isqrt(i - 1) + 1     # integer ceil-sqrt, as before
+
+
+def test_coverage_and_dense_equivalence_with_exponents_one_third_two_thirds():
+    """Span-length derivation of Section "Span attention" for general p: the gap between adjacent
+    anchors is (s+1)^(1/p) - s^(1/p) <= (1/p) (s+1)^(1/p - 1) <= (1/p) i^(1-p); with p = 1/3 and
+    l(i) = ceil(i^(2/3)) a backward factor of 3 covers every key, so attention over all anchors is
+    dense causal attention; a backward factor of 1 is not enough."""
+    B, Hq, Hkv, L, D = 1, 2, 1, 400, 8
+    q_s, q = rand((B, Hq, L, D), 13), rand((B, Hq, L, D), 14)
+    k, v = rand((B, Hkv, L, D), 15), rand((B, Hkv, L, D), 16)
+    sr = O.span_search(q_s, k, O.F64, top_k=10, search_exponent=1.0 / 3.0)
+    assert (sr["anchor"][0, 0, 399] >= 0).sum() == 7          # 1, 8, ..., 343 <= 400
+    at = O.span_attention(q, k, v, O.F64, sr["anchor"], span_len=0, back_factor=3, softmax_scale=0.3,
+                          span_exponent=2.0 / 3.0)
+    ref_out, ref_lse = dense_causal(q, k, v, 0.3)
+    np.testing.assert_allclose(at["out"], ref_out, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(at["lse"], ref_lse, rtol=0, atol=1e-12)
+    at1 = O.span_attention(q, k, v, O.F64, sr["anchor"], span_len=0, back_factor=1, softmax_scale=0.3,
+                           span_exponent=2.0 / 3.0)
+    assert at1["n_pairs"] < at["n_pairs"]
+
+
+def test_search_with_exponent_against_exhaustive_scoring():
+    B, Hq, Hkv, L, D, top_k = 1, 2, 2, 130, 8, 3
+    q_s, k = rand((B, Hq, L, D), 21), rand((B, Hkv, L, D), 22)
+    for p, root in ((1.0 / 3.0, 3), (0.25, 4)):
+        sr = O.span_search(q_s, k, O.F64, top_k=top_k, search_exponent=p)
+        for h in range(Hq):
+            for i in range(L):
+                cand = [i + 1 - m ** root for m in range(1, 12) if i + 1 - m ** root >= 0]
+                sc = np.array([q_s[0, h, i] @ k[0, h, t] for t in cand])
+                order = np.argsort(-sc, kind="stable")[:top_k]
+                want = [cand[j] for j in order] + [-1] * (top_k - len(order))
+                assert list(sr["anchor"][0, h, i]) == want
