@@ -98,6 +98,13 @@ typedef struct {
     int32_t mode;         /* sla_mode_t                                                           */
     float search_scale;   /* multiplies the search score (the paper's equation has none: 1.0f)    */
     float softmax_scale;  /* multiplies the attention logits ("scaled dot-product": 1/sqrt(D))     */
+    double search_exponent; /* p of the stride pattern (Section "Span attention", general p): the
+                              stride-s anchor of query i is i + 1 - ceil((s+1)^(1/p)); 0 or 0.5: the
+                              exact squares (s+1)^2; else 0.2 .. 0.8                             */
+    double span_exponent; /* with span_len = 0: l(i) = ceil(i^span_exponent); 0 or 0.5: the exact
+                              integer ceil(sqrt(i)); else 0.2 .. 0.8 (Section "Training": e.g. 1/3 for
+                              the search and 2/3 for the spans).  The powers are rounded up after
+                              taking off one part in 1e12, so that integer powers stay exact     */
 } sla_params_t;
 
 /* ---- handle ------------------------------------------------------------------------------- */

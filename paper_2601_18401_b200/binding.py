@@ -44,7 +44,8 @@ class sla_layout_t(C.Structure):
 class sla_params_t(C.Structure):
     _fields_ = [("top_k", C.c_int32), ("span_len", C.c_int32), ("back_factor", C.c_int32),
                 ("fwd_factor", C.c_int32), ("window", C.c_int32), ("mode", C.c_int32),
-                ("search_scale", C.c_float), ("softmax_scale", C.c_float)]
+                ("search_scale", C.c_float), ("softmax_scale", C.c_float),
+                ("search_exponent", C.c_double), ("span_exponent", C.c_double)]
 
 
 _lib = None
@@ -100,10 +101,12 @@ def load_library():
 
 def make_params(top_k: int, span_len: int, back_factor: int = 2, fwd_factor: int = 0, window: int = 0,
                 mode: int = SLA_UNION, search_scale: float = 1.0,
-                softmax_scale: Optional[float] = None, head_dim: int = 128) -> sla_params_t:
+                softmax_scale: Optional[float] = None, head_dim: int = 128,
+                search_exponent: float = 0.5, span_exponent: float = 0.5) -> sla_params_t:
     if softmax_scale is None:
         softmax_scale = 1.0 / math.sqrt(head_dim)
-    return sla_params_t(top_k, span_len, back_factor, fwd_factor, window, mode, search_scale, softmax_scale)
+    return sla_params_t(top_k, span_len, back_factor, fwd_factor, window, mode, search_scale, softmax_scale,
+                        search_exponent, span_exponent)
 
 
 def _dtype_code(t: torch.Tensor) -> int:

@@ -1,10 +1,12 @@
 // Host side of libsla: handle, argument validation, workspace carving and kernel dispatch.
 // Every exported function is declared and documented in include/sla.h.
+#include <math.h>
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "sla_kernels.h"
 
@@ -17,6 +19,11 @@ struct sla_handle_s {
     size_t scratch_avail = 0; // bytes of workspace after the header that kernels may use as scratch
     sla::KernelTimer timer;   // sla_set_kernel_timing / sla_kernel_time_ms
     bool force_simt = false;  // environment SLA_FORCE_SIMT=1: generic kernels only (for A/B checks)
+    // stride-offset and span-length tables for exponents other than 1/2 (host copies; the device
+    // copies sit in the workspace header) and what they were built for
+    std::vector<int> off_host, len_host;
+    double off_p = 0.0, len_p = 0.0;
+    long long off_reach = 0, len_reach = 0;
     // sla_prefill_host: copy-in and copy-out streams and per-chunk events, created on first use
     static constexpr int kMaxChunks = 16;
     cudaStream_t s_in = nullptr, s_out = nullptr;
@@ -26,8 +33,12 @@ struct sla_handle_s {
 
 namespace {
 
-// header of the workspace: status word at 0, completion counters of the decode step from byte 256
-constexpr size_t kHeaderBytes = 64 * 1024;
+// header of the workspace: status word at 0, completion counters of the decode step from byte 256,
+// then the two pattern tables (stride offsets, span-length steps) of kMaxTable ints each
+constexpr size_t kCounterEnd = 64 * 1024;
+constexpr int kMaxTable = 65536;
+constexpr size_t kOffTableAt = kCounterEnd, kLenTableAt = kCounterEnd + (size_t)kMaxTable * 4;
+constexpr size_t kHeaderBytes = kCounterEnd + 2 * (size_t)kMaxTable * 4;
 constexpr size_t kCounterOffset = 256;
 
 sla_status_t fail(sla_handle_t h, sla_status_t code, const char *fmt, const char *detail = "") {
@@ -63,7 +74,46 @@ const char *check_layout_params(const sla_layout_t *l, const sla_params_t *p, bo
     if (p->window < 0) return "window must be >= 0";
     if (p->mode != SLA_UNION && p->mode != SLA_PER_SPAN) return "mode must be SLA_UNION or SLA_PER_SPAN";
     if (!(p->softmax_scale == p->softmax_scale) || !(p->search_scale == p->search_scale)) return "scale is NaN";
+    for (double e : {p->search_exponent, p->span_exponent})
+        if (!(e == 0.0 || (e >= 0.2 && e <= 0.8))) return "exponents must be 0 (= 1/2) or in [0.2, 0.8]";
     return nullptr;
+}
+
+// ceil of base^expo, after taking off one part in 1e12: a power that is an integer in exact arithmetic
+// (exponent 1/3: cubes) must not be pushed to the next integer by the rounding of 1/p and of pow.
+long long ceil_pow(double base, double expo) {
+    const double x = pow(base, expo);
+    return (long long)ceil(x - 1e-12 * x);
+}
+
+bool is_half(double p) { return p == 0.0 || p == 0.5; }
+
+// off[s] = ceil((s+1)^(1/p)) for every stride whose offset is <= reach.  False when there are too many.
+bool build_offsets(double p, long long reach, std::vector<int> &off) {
+    off.clear();
+    for (long long s = 0;; ++s) {
+        const long long o = ceil_pow((double)(s + 1), 1.0 / p);
+        if (o > reach) break;
+        if ((int)off.size() >= kMaxTable) return false;
+        off.push_back((int)o);
+    }
+    return true;
+}
+
+// len_first[v-1] = smallest i >= 1 with ceil(i^p) >= v, for every v reached by some i <= reach.
+bool build_len_first(double p, long long reach, std::vector<int> &lf) {
+    lf.clear();
+    long long i = 1;
+    for (long long v = 1;; ++v) {
+        // l is non-decreasing and grows by at most 1 per position: start near (v-1)^(1/p) and settle
+        long long g = (long long)floor(pow((double)(v - 1), 1.0 / p)) - 2;
+        if (g > i) i = g;
+        while (i <= reach && ceil_pow((double)i, p) < v) ++i;
+        if (i > reach) break;
+        if ((int)lf.size() >= kMaxTable) return false;
+        lf.push_back((int)i);
+    }
+    return true;
 }
 
 // Kernels are launched on the current device: it has to be the one the handle was created on.
@@ -85,7 +135,43 @@ sla::Call make_call(const sla_handle_t h, const sla_layout_t *l, const sla_param
     c.window = p->window; c.mode = p->mode;
     c.search_scale = p->search_scale; c.softmax_scale = p->softmax_scale;
     c.status = h ? reinterpret_cast<int *>(h->ws) : nullptr;
+    c.off = c.off_host = c.len_first = c.len_first_host = nullptr;
+    c.n_off = c.n_len = 0;
+    if (h && !is_half(p->search_exponent)) {
+        c.off = reinterpret_cast<const int *>(h->ws + kOffTableAt);
+        c.off_host = h->off_host.data();
+        c.n_off = (int)h->off_host.size();
+    }
+    if (h && !is_half(p->span_exponent) && p->span_len == 0) {
+        c.len_first = reinterpret_cast<const int *>(h->ws + kLenTableAt);
+        c.len_first_host = h->len_host.data();
+        c.n_len = (int)h->len_host.size();
+    }
     return c;
+}
+
+// Builds (or reuses) the handle's pattern tables for this call's exponents and key range and puts
+// the device copies in place on `st`.  Must run before make_call.
+sla_status_t prepare_pattern(sla_handle_t h, const sla_params_t *p, int64_t Lkv, cudaStream_t st) {
+    if (!is_half(p->search_exponent) && (h->off_p != p->search_exponent || h->off_reach < Lkv)) {
+        if (!build_offsets(p->search_exponent, Lkv, h->off_host))
+            return fail(h, SLA_ERR_UNSUPPORTED, "search_exponent gives more than 65536 strides for this length%s");
+        h->off_p = p->search_exponent;
+        h->off_reach = Lkv;
+        if (!h->off_host.empty() &&
+            cudaMemcpyAsync(h->ws + kOffTableAt, h->off_host.data(), h->off_host.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return fail(h, SLA_ERR_CUDA, "copying the stride table failed%s");
+    }
+    if (!is_half(p->span_exponent) && p->span_len == 0 && (h->len_p != p->span_exponent || h->len_reach < Lkv)) {
+        if (!build_len_first(p->span_exponent, Lkv, h->len_host))
+            return fail(h, SLA_ERR_UNSUPPORTED, "span_exponent gives base lengths above 65536 for this length%s");
+        h->len_p = p->span_exponent;
+        h->len_reach = Lkv;
+        if (!h->len_host.empty() &&
+            cudaMemcpyAsync(h->ws + kLenTableAt, h->len_host.data(), h->len_host.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return fail(h, SLA_ERR_CUDA, "copying the span-length table failed%s");
+    }
+    return SLA_OK;
 }
 
 const char *check_prefill_range(int64_t Lq, int64_t q_pos0, int64_t Lkv) {
@@ -111,7 +197,8 @@ sla_status_t check_decode_args(const void *q_s, const void *q, const void *k_cac
     if (!q_s || !q || !k_cache || !v_cache || !out || !lse || !out_anchor || !out_score) return SLA_ERR_INVALID_ARG;
     if (!aligned16(q_s) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
         return SLA_ERR_INVALID_ARG;
-    if (p->window != 0 || p->mode != SLA_UNION) return SLA_ERR_UNSUPPORTED;
+    if (p->window != 0 || p->mode != SLA_UNION || !is_half(p->search_exponent) || !is_half(p->span_exponent))
+        return SLA_ERR_UNSUPPORTED;
     *c_out = make_call(nullptr, l, p, 1, n_ctx - 1, n_ctx);
     return SLA_OK;
 }
@@ -212,6 +299,17 @@ sla_status_t sla_destroy(sla_handle_t h) {
 size_t sla_workspace_bytes(const sla_layout_t *l, const sla_params_t *p, int64_t Lq, int64_t Lkv) {
     if (check_layout_params(l, p, true) || Lq <= 0 || Lkv <= 0 || Lq > Lkv) return 0;
     sla::Call c = make_call(nullptr, l, p, Lq, Lkv - Lq, Lkv);
+    std::vector<int> off, lf;   // host tables for the plans below, when the exponents are not 1/2
+    if (!is_half(p->search_exponent)) {
+        if (!build_offsets(p->search_exponent, Lkv, off)) return 0;
+        c.off_host = off.data();
+        c.n_off = (int)off.size();
+    }
+    if (!is_half(p->span_exponent) && p->span_len == 0) {
+        if (!build_len_first(p->span_exponent, Lkv, lf)) return 0;
+        c.len_first_host = lf.data();
+        c.n_len = (int)lf.size();
+    }
     // the SM count only changes how the decode work is split; size for a generous upper bound
     const sla::DecodePlan dp = sla::plan_decode(c, Lkv, 256 * l->batch * l->n_q_heads);
     size_t need = dp.bytes;
@@ -245,6 +343,7 @@ sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int
     if (!q_s || !k || !out_anchor || !out_score) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
     if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!aligned16(q_s) || !aligned16(k)) return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
+    if (sla_status_t ps = prepare_pattern(h, p, Lkv, static_cast<cudaStream_t>(stream))) return ps;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!h->force_simt && sla::search_mma_supported(c, l->dtype)) {
@@ -270,6 +369,7 @@ sla_status_t span_attention_impl(sla_handle_t h, const void *q, const void *k, c
     if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
         return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
+    if (sla_status_t ps = prepare_pattern(h, p, Lkv, static_cast<cudaStream_t>(stream))) return ps;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!h->force_simt && sla::tc_attention_supported(c, l->dtype)) {
@@ -326,13 +426,14 @@ sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, con
         return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
     if (!aligned16(q_s) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
         return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
+    if (sla_status_t ps = prepare_pattern(h, p, n_ctx, static_cast<cudaStream_t>(stream))) return ps;
     sla::Call c = make_call(h, l, p, 1, n_ctx - 1, n_ctx);
     const sla::DecodePlan plan =
         sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim));
     if (plan.bytes + kHeaderBytes > h->ws_bytes) return fail(h, SLA_ERR_WORKSPACE, "workspace too small for this decode step%s");
     if ((size_t)plan.n_anchor * sizeof(float) * 8 > 180 * 1024) return fail(h, SLA_ERR_UNSUPPORTED, "context too long for the decode top-k stage%s");
     const size_t units = p->mode == SLA_PER_SPAN ? (size_t)p->top_k : 1;
-    if ((size_t)(l->batch) * (l->n_kv_heads + l->n_q_heads * (units + 1)) * sizeof(int) > kHeaderBytes - kCounterOffset)
+    if ((size_t)(l->batch) * (l->n_kv_heads + l->n_q_heads * (units + 1)) * sizeof(int) > kCounterEnd - kCounterOffset)
         return fail(h, SLA_ERR_UNSUPPORTED, "too many (batch, head) pairs for the decode step%s");
     cudaError_t e = sla::launch_decode(q_s, q, k_cache, v_cache, c, l->dtype, n_ctx, plan, h->ws + kHeaderBytes,
                                        reinterpret_cast<int *>(h->ws + kCounterOffset), out, lse, out_anchor,

@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
         const int h = g * a.G + hg;
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
         const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
-        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len), a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
+        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len, a.len_first, a.n_len), a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
         if (PASS == 0) a.n_pieces[((long long)b * a.Hq + h) * a.Lc + rc] = (unsigned char)cnt;
         for (int j = 0; j < cnt; ++j) atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
     }
@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
         const int h = g * a.G + hg;
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
         const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
-        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len), a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
+        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len, a.len_first, a.n_len), a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
         const int row = (int)(((long long)b * a.Hq + h) * a.Lc + rc);
         for (int j = 0; j < cnt; ++j) {
             const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);

@@ -648,7 +648,7 @@ tc_merge_gated(const __half *__restrict__ part_o, const float2 *__restrict__ par
     const int32_t *an = anchor + orow * c.top_k;
     const float *sc = score + orow * c.top_k;
     const float2 *pl = part_lse + row * slots;
-    const long long ell = base_len(i, c.span_len);
+    const long long ell = base_len(c, i);
     const long long w_lo = i - c.window + 1 > 0 ? i - c.window + 1 : 0;
     const bool has_w = c.window > 0;
     const float lw = has_w ? pl[c.top_k].x : -CUDART_INF_F;
@@ -780,7 +780,7 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 bool tc_attention_shape_ok(const Call &c, int dtype) {
     if (dtype != SLA_BF16 || c.D != kD) return false;
     if (c.kv_st < kD || c.top_k > kMaxTopK || !(c.softmax_scale > 0.f)) return false;
-    const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
+    const long long ell = base_len(c, c.q_pos0 + c.Lq - 1);
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     if (c.window > span_tokens) span_tokens = c.window;
     return span_tokens / kBK + 2 <= 4096;
@@ -796,7 +796,7 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     p.Lc = Lc;
     p.n_bg = c.B * c.Hkv;
     p.NB = (int)((c.Lkv + kBK - 1) / kBK);
-    const long long ell = base_len(c.q_pos0 + c.Lq - 1, c.span_len);
+    const long long ell = base_len(c, c.q_pos0 + c.Lq - 1);
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     if (c.window > span_tokens) span_tokens = c.window;   // the window is a piece too
     if (span_tokens > c.Lkv) span_tokens = c.Lkv;
@@ -860,7 +860,7 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         tc::PrepArgs pa;
         pa.anchor = anchor; pa.B = c.B; pa.Hq = c.Hq; pa.Hkv = c.Hkv; pa.G = c.G; pa.top_k = c.top_k;
         pa.span_len = c.span_len; pa.back = c.back; pa.fwd = c.fwd; pa.Lq = c.Lq; pa.q_pos0 = c.q_pos0;
-        pa.window = c.window; pa.mode = c.mode;
+        pa.window = c.window; pa.mode = c.mode; pa.len_first = c.len_first; pa.n_len = c.n_len;
         pa.r0 = r0; pa.Lc = lc; pa.NB = plan.NB; pa.nb_max = plan.nb_max; pa.ncls = plan.ncls;
         pa.ctas_per_bg = plan.ctas_per_bg;
         pa.key_count = (int *)(ws + plan.off_key_count);

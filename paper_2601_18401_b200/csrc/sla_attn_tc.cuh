@@ -19,6 +19,8 @@ struct PrepArgs {
     const int32_t *anchor;   // [B,Hq,Lq,top_k]
     int B, Hq, Hkv, G, top_k, span_len, back, fwd;
     int window, mode;        // local window w (0 = none); sla_mode_t
+    const int *len_first;    // steps of l(i) for a span exponent other than 1/2 (device), else NULL
+    int n_len;
     long long Lq, q_pos0, r0;
     int Lc;                  // query positions in this chunk
     int NB;                  // 64-key blocks in [0, Lkv)

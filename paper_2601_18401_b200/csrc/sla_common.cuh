@@ -25,6 +25,14 @@ struct Call {
     int window, mode;               // local window w (0 = none); sla_mode_t
     float search_scale, softmax_scale;
     int *status;                    // device status word
+    // Exponents other than 1/2 (Section "Span attention", general p; Section "Training"): the stride
+    // offsets and the span-length steps come from tables the host builds (NULL: the exact integer
+    // rules for p = 1/2).  off[s] = ceil((s+1)^(1/p_search)), ascending; len_first[v-1] = smallest i
+    // with l(i) = ceil(i^p_span) >= v.  The *_host copies serve the host-side plans.
+    const int *off, *off_host;
+    int n_off;
+    const int *len_first, *len_first_host;
+    int n_len;
 };
 
 // floor(sqrt(x)) for 0 <= x < 2^62, exact.
@@ -36,12 +44,59 @@ __host__ __device__ inline long long isqrt_ll(long long x) {
     return r;
 }
 
-// Base span length l(i) (Algorithm 1: l(i) = ceil(sqrt(i)) unless a fixed length is given).
-__host__ __device__ inline long long base_len(long long i, int span_len) {
+// Number of entries of the ascending table a[0..n) that are <= x.
+__host__ __device__ inline int count_le(const int *a, int n, long long x) {
+    int lo = 0, hi = n;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (a[mid] <= x) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// Base span length l(i) (Algorithm 1: l(i) = ceil(sqrt(i)) unless a fixed length is given; with a
+// span exponent other than 1/2 the steps of ceil(i^p) come from the table).
+__host__ __device__ inline long long base_len(long long i, int span_len, const int *len_first = nullptr,
+                                              int n_len = 0) {
     if (span_len > 0) return span_len;
     if (i <= 0) return 0;
+    if (len_first) return count_le(len_first, n_len, i);
     long long r = isqrt_ll(i);
     return r * r < i ? r + 1 : r;
+}
+
+// Stride pattern of a call.  In device code the device tables are read, in host code the host copies.
+__host__ __device__ inline const int *pattern_off(const Call &c) {
+#ifdef __CUDA_ARCH__
+    return c.off;
+#else
+    return c.off_host;
+#endif
+}
+__host__ __device__ inline const int *pattern_len(const Call &c) {
+#ifdef __CUDA_ARCH__
+    return c.len_first;
+#else
+    return c.len_first_host;
+#endif
+}
+// Strides whose anchor exists for query position i: offsets <= i + 1.
+__host__ __device__ inline int n_strides(const Call &c, long long i) {
+    const int *off = pattern_off(c);
+    return off ? count_le(off, c.n_off, i + 1) : (int)isqrt_ll(i + 1);
+}
+// Strides whose anchor lies inside the local window: offsets <= w.
+__host__ __device__ inline int window_strides(const Call &c) {
+    const int *off = pattern_off(c);
+    return off ? count_le(off, c.n_off, c.window) : (int)isqrt_ll(c.window);
+}
+// Distance of the stride-s anchor from position i + 1.
+__host__ __device__ inline int stride_offset(const Call &c, int s) {
+    const int *off = pattern_off(c);
+    return off ? off[s] : (s + 1) * (s + 1);
+}
+__host__ __device__ inline long long base_len(const Call &c, long long i) {
+    return base_len(i, c.span_len, pattern_len(c), c.n_len);
 }
 
 // ---- element loads: a 16-byte vector of T widened to fp32 ------------------------------------

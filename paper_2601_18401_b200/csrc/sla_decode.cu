@@ -67,7 +67,7 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
         for (int t = 0; t < GT; ++t) part[u][t] = 0.f;
         if (s < n) {
             // candidate x is stride s_min + x: the first s_min strides land inside the local window
-            const long long tpos = i + 1 - (long long)(s_min + s + 1) * (s_min + s + 1);
+            const long long tpos = i + 1 - stride_offset(c, s_min + s);
             float kv[E];
             Vec16<T>::load(kbase + tpos * c.kv_st + sub * E, kv);
 #pragma unroll
@@ -105,7 +105,7 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
     float *cand_v = sc + n;
     int *cand_s = reinterpret_cast<int *>(cand_v + topk::kCap);
     int *s_lo = cand_s + topk::kCap, *s_hi = s_lo + kIv, *p_lo = s_hi + kIv, *p_hi = p_lo + kIv;
-    const long long ell = base_len(i, c.span_len);
+    const long long ell = base_len(c, i);
     // span table of an attention unit: piece starts [pcap], cumulative token counts [pcap + 1], count
     const int pcap = c.mode == SLA_PER_SPAN ? 2 : c.top_k + 1, tstride = 2 * pcap + 2;
     for (int hg = warp; hg < c.G; hg += kWarps) {
@@ -114,7 +114,7 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
         for (int s = lane; s < n; s += 32) sc[s] = __ldcg(src + s);   // written by other SMs: bypass L1
         __syncwarp();
         topk::select_topk(sc, n, c.top_k, i, cand_v, cand_s, out_anchor + bh * c.top_k, out_score + bh * c.top_k, lane,
-                          s_min);
+                          s_min, c.off);
         __syncwarp();
         // intervals: the spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)])
         // and, last, the local window W = [max(0, i-w+1), i]
@@ -438,7 +438,7 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
     float *unit_out = (float *)(base + p.off_unit_out);
     const int units = c.mode == SLA_PER_SPAN ? c.top_k : 1;
     int *done_bg = counters, *done_unit = counters + c.B * c.Hkv, *done_head = done_unit + c.B * c.Hq * units;
-    const int n = p.n_anchor, s_min = (int)isqrt_ll(c.window);
+    const int n = p.n_anchor, s_min = window_strides(c);
     const int rows_per_cta = (kScoreThreads / 32) * RPI * 2;
     const int gt = c.G % 8 == 0 ? 8 : c.G % 4 == 0 ? 4 : c.G % 2 == 0 ? 2 : 1;
     dim3 gs(n > 0 ? (n + rows_per_cta - 1) / rows_per_cta : 1, c.B * c.Hkv, c.G / gt);
@@ -491,9 +491,9 @@ int decode_attn_blocks_per_sm(int dtype, int D) {
 DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots) {
     DecodePlan p;
     // candidates: the strides whose anchor lies left of the local window
-    const long long n_cand = isqrt_ll(n_ctx) - isqrt_ll(c.window);
+    const long long n_cand = n_strides(c, n_ctx - 1) - window_strides(c);
     p.n_anchor = (int)(n_cand > 0 ? n_cand : 0);
-    const long long ell = base_len(n_ctx - 1, c.span_len);
+    const long long ell = base_len(c, n_ctx - 1);
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     if (span_tokens > n_ctx) span_tokens = n_ctx;
     const bool per_span = c.mode == SLA_PER_SPAN;

@@ -46,9 +46,9 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
     if (r >= c.Lq) return;
     const int bg = blockIdx.y, g = bg % c.Hkv, b = bg / c.Hkv;
     const long long i = c.q_pos0 + r;
-    const int n = (int)isqrt_ll(i + 1);
+    const int n = n_strides(c, i);
     // Algorithm 1: anchors inside the local window are no candidates; t_s lies in W iff (s+1)^2 <= w
-    const int s_min = (int)isqrt_ll(c.window);
+    const int s_min = window_strides(c);
     float *sc = smem + (size_t)warp * (heads * n_max + 2 * kCap);
     float *cand_v = sc + heads * n_max;
     int *cand_s = reinterpret_cast<int *>(cand_v + kCap);
@@ -70,8 +70,8 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
     const int kv_st = (int)c.kv_st, i32 = (int)i;   // positions and the token stride fit 31 bits: 32x32->64 products
     for (int a0 = s_min; a0 < n; a0 += 16) {
         const int s0 = a0 + r8, s1 = s0 + 8;
-        const int t0 = s0 < n ? i32 + 1 - (s0 + 1) * (s0 + 1) : i32;
-        const int t1 = s1 < n ? i32 + 1 - (s1 + 1) * (s1 + 1) : i32;
+        const int t0 = s0 < n ? i32 + 1 - stride_offset(c, s0) : i32;
+        const int t1 = s1 < n ? i32 + 1 - stride_offset(c, s1) : i32;
         const bf16 *row0 = kbase + (long long)t0 * kv_st, *row1 = kbase + (long long)t1 * kv_st;
         uint4 ra[4], rb[4];
 #pragma unroll
@@ -100,7 +100,7 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
         const int h = g * c.G + head0 + hh;
         const long long obase = ((((long long)b * c.Hq + h) * c.Lq) + r) * c.top_k;
         select_topk(sc + hh * n_max, n > s_min ? n - s_min : 0, c.top_k, i, cand_v, cand_s, out_anchor + obase,
-                    out_score + obase, lane, s_min);
+                    out_score + obase, lane, s_min, c.off);
     }
 }
 
@@ -108,14 +108,14 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
 
 bool search_mma_supported(const Call &c, int dtype) {
     if (dtype != SLA_BF16 || c.D != 128 || (long long)c.B * c.Hkv > 65535 || c.kv_st > INT_MAX) return false;
-    const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
+    const int n_max = n_strides(c, c.q_pos0 + c.Lq - 1) + 1;
     const int heads = c.G < 8 ? c.G : 8;
     return (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float) <= 200 * 1024;
 }
 
 cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int32_t *oa, float *os, cudaStream_t st,
                               long long *launches) {
-    const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
+    const int n_max = n_strides(c, c.q_pos0 + c.Lq - 1) + 1;
     const dim3 blocks((unsigned)((c.Lq + kWarps - 1) / kWarps), (unsigned)(c.B * c.Hkv));
     for (int head0 = 0; head0 < c.G; head0 += 8) {
         const int heads = c.G - head0 < 8 ? c.G - head0 : 8;

@@ -60,8 +60,8 @@ search_rows_simt(const T *__restrict__ q_s, const T *__restrict__ k, Call c,
     const RowId id = decode_row(row, c);
     const long long i = c.q_pos0 + id.r;
     // Algorithm 1: T = Anchors(i) without the window; t_s lies in W exactly when (s+1)^2 <= w
-    const int s_min = (int)isqrt_ll(c.window);
-    const int n = (int)isqrt_ll(i + 1);
+    const int s_min = window_strides(c);
+    const int n = n_strides(c, i);
     float *sc = smem + (size_t)warp * n_max;
     const T *qrow = q_s + id.b * c.q_sb + id.h * c.q_sh + id.r * c.q_st;
     const T *kbase = k + id.b * c.kv_sb + id.g * c.kv_sh;
@@ -77,7 +77,7 @@ search_rows_simt(const T *__restrict__ q_s, const T *__restrict__ k, Call c,
             const int s = s0 + u * RPI + rsel;
             part[u] = 0.f;
             if (s < n) {
-                const long long t = i + 1 - (long long)(s + 1) * (s + 1);
+                const long long t = i + 1 - stride_offset(c, s);
                 float kv[E];
                 Vec16<T>::load(kbase + t * c.kv_st + sub * E, kv);
 #pragma unroll
@@ -109,7 +109,7 @@ search_rows_simt(const T *__restrict__ q_s, const T *__restrict__ k, Call c,
         }
         if (lane == 0) {
             if (bs != INT_MAX) {
-                out_anchor[obase + j] = (int32_t)(i + 1 - (long long)(bs + 1) * (bs + 1));
+                out_anchor[obase + j] = (int32_t)(i + 1 - stride_offset(c, bs));
                 out_score[obase + j] = bv;
                 sc[bs] = -CUDART_INF_F;
             } else {
@@ -218,7 +218,7 @@ attn_rows_simt(const T *__restrict__ q, const T *__restrict__ k, const T *__rest
     if (row >= (long long)c.B * c.Hq * c.Lq) return;
     const RowId id = decode_row(row, c);
     const long long i = c.q_pos0 + id.r;
-    const long long ell = base_len(i, c.span_len);
+    const long long ell = base_len(c, i);
     const long long orow_idx = (((long long)id.b * c.Hq + id.h) * c.Lq) + id.r;
     const long long abase = orow_idx * c.top_k;
     const int n_iv = c.top_k + (c.window > 0 ? 1 : 0);
@@ -372,7 +372,7 @@ template <typename T, int D>
 cudaError_t search_launch(const void *q_s, const void *k, const Call &c, int32_t *oa, float *os,
                           cudaStream_t st) {
     const long long rows = (long long)c.B * c.Hq * c.Lq;
-    const int n_max = (int)isqrt_ll(c.q_pos0 + c.Lq) + 1;
+    const int n_max = n_strides(c, c.q_pos0 + c.Lq - 1) + 1;
     const size_t smem = (size_t)kWarpsPerBlock * n_max * sizeof(float);
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
     auto kern = search_rows_simt<T, D>;

@@ -18,9 +18,11 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 
 // Top-k of sc[0..n) for one head, sc[x] being the score of stride index s_base + x (the strides
 // below s_base have their anchors inside the local window and are no candidates); writes
-// anchors/scores.  All lanes of the warp take part.
+// anchors/scores.  `off`, when not NULL, is the table of stride offsets (else (s+1)^2).  All lanes of
+// the warp take part.
 __device__ inline void select_topk(float *sc, int n, int top_k, long long i, float *cand_v, int *cand_s,
-                            int32_t *out_anchor, float *out_score, int lane, int s_base = 0) {
+                            int32_t *out_anchor, float *out_score, int lane, int s_base = 0,
+                            const int *off = nullptr) {
     const uint32_t kNegInfKey = order_key(-CUDART_INF_F);
     // A. lane maxima over the strided slots
     float lm = -CUDART_INF_F;
@@ -66,7 +68,7 @@ __device__ inline void select_topk(float *sc, int n, int top_k, long long i, flo
             }
             if (rank < top_k) {
                 const long long m = s_base + sc_ + 1;
-                out_anchor[rank] = (int32_t)(i + 1 - m * m);
+                out_anchor[rank] = (int32_t)(i + 1 - (off ? (long long)off[m - 1] : m * m));
                 out_score[rank] = __uint_as_float((kc & 0x80000000u) ? (kc & 0x7fffffffu) : ~kc);
             }
         }
@@ -91,7 +93,8 @@ __device__ inline void select_topk(float *sc, int n, int top_k, long long i, flo
             }
             if (lane == 0) {
                 if (bs != INT_MAX) {
-                    out_anchor[j] = (int32_t)(i + 1 - (long long)(s_base + bs + 1) * (s_base + bs + 1));
+                    out_anchor[j] = (int32_t)(i + 1 - (off ? (long long)off[s_base + bs]
+                                                            : (long long)(s_base + bs + 1) * (s_base + bs + 1)));
                     out_score[j] = bv;
                     sc[bs] = -CUDART_INF_F;
                 } else {

@@ -131,3 +131,92 @@ def test_decode_modes_and_window(sla, handle, mode, window, n_ctx0, span_len, to
                                score=score.cpu().numpy().astype(np.float64)[:, :, None],
                                q_pos0=n_ctx - 1, Lkv=n_ctx)
         P.compare_attention(out[:, :, None], lse[:, :, None], att, dtype)
+
+
+def run_exponents(sla, handle, w, p_search, p_span, window=0, mode="union", top_k=None, back=2):
+    """Search + attention with general exponents (anchors at i + 1 - ceil((s+1)^(1/p)), base length
+    ceil(i^p_span)) against the oracle with the same exponents."""
+    from paper_2601_18401_b200 import synth
+    x = synth.make_prefill(w, device="cuda:0")
+    host = P.host_inputs(x)
+    code = synth.dtype_code(w.dtype)
+    k_sel = top_k or w.top_k
+    m_gpu = sla.SLA_PER_SPAN if mode == "per_span" else sla.SLA_UNION
+    m_ref = O.PER_SPAN if mode == "per_span" else O.UNION
+    params = sla.make_params(k_sel, w.span_len, back, w.fwd_factor, window=window, mode=m_gpu,
+                             head_dim=w.head_dim, search_exponent=p_search, span_exponent=p_span)
+    anchor, score = sla.sla_span_search(handle, x["q_s"], x["k"], params)
+    torch.cuda.synchronize()
+    ref_s = O.span_search(host["q_s"], host["k"], code, top_k=k_sel, window=window, search_exponent=p_search)
+    a, ra = anchor.cpu().numpy(), ref_s["anchor"]
+    clear = ref_s["gap"] > P.TIE_GAP
+    same = np.all(np.sort(a, axis=-1) == np.sort(ra, axis=-1), axis=-1)
+    assert not (~same & clear).any(), "selected anchors differ on clear-cut rows"
+    # every selected anchor sits on the stride pattern
+    offs = {O.stride_offset(s, p_search) for s in range(O.n_strides(w.seq_len, p_search) + 1)}
+    d = (np.arange(w.seq_len)[None, None, :, None] + 1 - a.astype(np.int64))[a >= 0]
+    assert set(np.unique(d).tolist()) <= offs
+    kw = dict(span_len=w.span_len, back_factor=back, fwd_factor=w.fwd_factor, window=window, mode=m_ref,
+              span_exponent=p_span, score=score.cpu().numpy().astype(np.float64))
+    ref_a = O.span_attention(host["q"], host["k"], host["v"], code, np.ascontiguousarray(a), **kw)
+    if mode == "per_span":
+        out, lse, _ = sla.sla_span_attention_gated(handle, x["q"], x["k"], x["v"], anchor, score, params)
+    else:
+        out, lse = sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    P.compare_attention(out, lse, ref_a, w.dtype)
+    return anchor, out, lse
+
+
+@pytest.mark.parametrize("p_search,p_span", [(1.0 / 3.0, 2.0 / 3.0), (0.54, 0.54), (0.4, 0.5), (0.5, 0.6)])
+@pytest.mark.parametrize("kw", [
+    dict(span_len=0, top_k=3),                                          # bf16 D128 GQA, l(i) from the exponent
+    dict(span_len=0, dtype="f32", head_dim=64, n_q_heads=2, n_kv_heads=1, seq_len=600, top_k=2),
+    dict(span_len=12, top_k=4),                                         # fixed base length
+])
+def test_general_exponents(sla, handle, kw, p_search, p_span):
+    run_exponents(sla, handle, workload(**kw), p_search, p_span)
+
+
+def test_general_exponents_with_window_and_gate(sla, handle):
+    run_exponents(sla, handle, workload(span_len=0, top_k=2, seq_len=1500), 1.0 / 3.0, 2.0 / 3.0, window=100,
+                  mode="per_span", back=3)
+    run_exponents(sla, handle, workload(span_len=0, top_k=2, seq_len=900), 0.54, 0.54, window=64, mode="union")
+
+
+def test_exponents_one_third_two_thirds_cover_everything(sla, handle):
+    """All anchors selected, p = (1/3, 2/3), backward factor 3: the union attends to every key, so the
+    result is dense causal attention (the coverage argument of Section "Span attention" for general p)."""
+    from paper_2601_18401_b200 import synth
+    w = workload(span_len=0, top_k=12, seq_len=900, n_q_heads=2, n_kv_heads=1)
+    anchor, out, lse = run_exponents(sla, handle, w, 1.0 / 3.0, 2.0 / 3.0, back=3)
+    x = synth.make_prefill(w, device="cuda:0")
+    q, k, v = x["q"].float(), x["k"].float(), x["v"].float()
+    k, v = k.repeat_interleave(2, dim=1), v.repeat_interleave(2, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True)
+    assert (out.float() - ref).abs().max().item() <= P.OUT_TOL["bf16"]
+
+
+def test_decode_with_general_exponents(sla, handle):
+    from paper_2601_18401_b200 import synth
+    w = synth.Workload("de", "decode", 1, 8, 2, 128, 4000, "bf16", 0, 3, seed=93)
+    kc, vc = synth.make_decode_cache(w, "cuda:0", capacity=4002)
+    hk, hv = synth.to_numpy(kc), synth.to_numpy(vc)
+    code = synth.dtype_code("bf16")
+    for p_search, p_span, back in ((1.0 / 3.0, 2.0 / 3.0, 3), (0.54, 0.54, 2)):
+        params = sla.make_params(3, 0, back, head_dim=128, search_exponent=p_search, span_exponent=p_span)
+        x = synth.make_decode_step_inputs(w, 0, "cuda:0")
+        n_ctx = 4001
+        kc[:, :, n_ctx - 1] = x["k_new"]; vc[:, :, n_ctx - 1] = x["v_new"]
+        hk[:, :, n_ctx - 1] = synth.to_numpy(x["k_new"]); hv[:, :, n_ctx - 1] = synth.to_numpy(x["v_new"])
+        out, lse, anchor, score = sla.sla_decode_step(handle, x["q_s"], x["q"], kc, vc, n_ctx, params)
+        torch.cuda.synchronize()
+        ref = O.decode_step(synth.to_numpy(x["q_s"]), synth.to_numpy(x["q"]), hk, hv, code, n_ctx=n_ctx, top_k=3,
+                            span_len=0, back_factor=back, search_exponent=p_search, span_exponent=p_span)
+        clear = ref["gap"] > P.TIE_GAP
+        same = np.all(np.sort(anchor.cpu().numpy(), -1) == np.sort(ref["anchor"], -1), axis=-1)
+        assert not (~same & clear).any()
+        att = O.span_attention(synth.to_numpy(x["q"])[:, :, None], hk, hv, code, anchor.cpu().numpy()[:, :, None],
+                               span_len=0, back_factor=back, q_pos0=n_ctx - 1, Lkv=n_ctx, span_exponent=p_span)
+        P.compare_attention(out[:, :, None], lse[:, :, None], att, "bf16")
