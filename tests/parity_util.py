@@ -48,27 +48,51 @@ def compare_search(anchor_gpu, score_gpu, ref, q_pos0=0, rows=None):
     return int((~clear).sum())
 
 
-def oracle_attention_for(x_host, dtype_code, anchor_gpu, w, q_pos0=0, rows=None, softmax_scale=None):
-    if rows is not None:
-        anchor_gpu = anchor_gpu[:, :, torch.as_tensor(np.asarray(rows), device=anchor_gpu.device)]
-    a = np.ascontiguousarray(anchor_gpu.cpu().numpy())
+def oracle_attention_for(x_host, dtype_code, anchor_ref, w, q_pos0=0, rows=None, softmax_scale=None):
+    """Oracle span-attention on anchors that come from the oracle's own search (or from the test's own
+    generator): nothing the CUDA path produced is ever an input of the oracle.  With `rows`,
+    anchor_ref holds those rows only."""
+    a = np.ascontiguousarray(np.asarray(anchor_ref), dtype=np.int32)
     return O.span_attention(x_host["q"], x_host["k"], x_host["v"], dtype_code, a, span_len=w.span_len,
                             back_factor=w.back_factor, fwd_factor=w.fwd_factor, q_pos0=q_pos0, rows=rows,
                             softmax_scale=softmax_scale)
 
 
-def compare_attention(out_gpu, lse_gpu, ref, dtype_name, rows=None):
+def oracle_anchors_on_device(anchor_gpu, ref_s, rows=None):
+    """The anchors the CUDA attention is given in a parity test: the oracle's selection (on all rows,
+    or written over the sampled `rows` of the CUDA search result, which fills the rest)."""
+    ra = torch.from_numpy(np.ascontiguousarray(ref_s["anchor"])).to(anchor_gpu.device)
+    if rows is None:
+        return ra.contiguous()
+    a = anchor_gpu.clone()
+    a[:, :, torch.as_tensor(np.asarray(rows), device=a.device)] = ra
+    return a
+
+
+def same_selection(anchor_gpu, ref_anchor):
+    """Rows on which the CUDA search and the oracle selected the same anchors (as sets)."""
+    a = anchor_gpu.cpu().numpy() if torch.is_tensor(anchor_gpu) else np.asarray(anchor_gpu)
+    return np.all(np.sort(a, axis=-1) == np.sort(ref_anchor, axis=-1), axis=-1)
+
+
+def compare_attention(out_gpu, lse_gpu, ref, dtype_name, rows=None, where=None):
+    """`where`: optional boolean mask [B,Hq,R] of the rows to compare (default all)."""
     if rows is not None:
         idx = torch.as_tensor(np.asarray(rows), device=out_gpu.device)
         out_gpu, lse_gpu = out_gpu[:, :, idx], lse_gpu[:, :, idx]
     o = out_gpu.float().cpu().numpy().astype(np.float64)
     l = lse_gpu.cpu().numpy().astype(np.float64)
+    ro, rl = ref["out"], ref["lse"]
+    if where is not None:
+        o, l, ro, rl = o[where], l[where], ro[where], rl[where]
+        if o.size == 0:
+            return 0.0, 0.0
     tol = OUT_TOL[dtype_name]
-    err = np.abs(o - ref["out"]).max()
+    err = np.abs(o - ro).max()
     assert err <= tol, f"output max-abs error {err} above {tol}"
-    fin = np.isfinite(ref["lse"])
+    fin = np.isfinite(rl)
     assert np.array_equal(np.isneginf(l), ~fin)
-    lerr = np.abs(l[fin] - ref["lse"][fin]).max() if fin.any() else 0.0
+    lerr = np.abs(l[fin] - rl[fin]).max() if fin.any() else 0.0
     assert lerr <= LSE_TOL[dtype_name], f"lse max-abs error {lerr}"
     return float(err), float(lerr)
 

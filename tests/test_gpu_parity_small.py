@@ -41,14 +41,17 @@ def run_prefill(sla, handle, w, q_pos0=0, Lq=None, permute=False, softmax_scale=
     q_s = x["q_s"][:, :, q_pos0:q_pos0 + Lq]
     q = x["q"][:, :, q_pos0:q_pos0 + Lq]
     anchor, score = sla.sla_span_search(handle, q_s, x["k"], params, q_pos0=q_pos0)
-    out, lse = sla.sla_span_attention(handle, q, x["k"], x["v"], anchor, params, q_pos0=q_pos0)
     torch.cuda.synchronize()
-    assert sla.sla_poll_status(handle) == sla.SLA_OK
     host = P.host_inputs({"q_s": q_s, "q": q, "k": x["k"], "v": x["v"]})
     code = synth.dtype_code(w.dtype)
     ref_s = O.span_search(host["q_s"], host["k"], code, top_k=w.top_k, q_pos0=q_pos0, search_scale=search_scale)
     ties = P.compare_search(anchor, score, ref_s, q_pos0=q_pos0)
-    ref_a = P.oracle_attention_for(host, code, anchor, w, q_pos0=q_pos0, softmax_scale=softmax_scale)
+    # the attention runs on the oracle's selection, on both sides
+    anchor = P.oracle_anchors_on_device(anchor, ref_s)
+    out, lse = sla.sla_span_attention(handle, q, x["k"], x["v"], anchor, params, q_pos0=q_pos0)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    ref_a = P.oracle_attention_for(host, code, ref_s["anchor"], w, q_pos0=q_pos0, softmax_scale=softmax_scale)
     err, lerr = P.compare_attention(out, lse, ref_a, w.dtype)
     return dict(ties=ties, err=err, lerr=lerr, anchor=anchor, out=out, lse=lse, host=host, ref_a=ref_a)
 
@@ -114,7 +117,7 @@ def test_attention_with_foreign_anchors(sla, handle):
     out, lse = sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params)
     torch.cuda.synchronize()
     assert sla.sla_poll_status(handle) == sla.SLA_OK
-    ref = P.oracle_attention_for(P.host_inputs(x), O.BF16, anchor, w)
+    ref = P.oracle_attention_for(P.host_inputs(x), O.BF16, anchor.cpu().numpy(), w)   # the test's own anchors
     P.compare_attention(out, lse, ref, "bf16")
     assert torch.all(out[:, :, 100:120] == 0) and torch.all(torch.isinf(lse[:, :, 100:120]))
     # an anchor beyond the query position is skipped and reported, never dereferenced
@@ -143,13 +146,12 @@ def test_decode_parity(sla, handle, dtype, D, Hq, Hkv):
                             n_ctx=n_ctx, top_k=top_k, span_len=span_len)
         rs = {k_: ref[k_][:, :, None] for k_ in ("anchor", "score", "gap")}
         P.compare_search(anchor[:, :, None], score[:, :, None], rs, q_pos0=n_ctx - 1)
-        ref2 = O.decode_step(synth.to_numpy(step["q_s"]), synth.to_numpy(step["q"]), hk, hv, code,
-                             n_ctx=n_ctx, top_k=top_k, span_len=span_len)
-        # attention parity on the GPU's own anchors
-        att = O.span_attention(synth.to_numpy(step["q"])[:, :, None], hk, hv, code,
-                               anchor.cpu().numpy()[:, :, None], span_len=span_len, q_pos0=n_ctx - 1, Lkv=n_ctx)
-        P.compare_attention(out[:, :, None], lse[:, :, None], att, dtype)
-        del ref2
+        # the step's output against the oracle's own step, on the heads where both selected the same
+        # anchors (the others are near-ties, counted by compare_search)
+        same = P.same_selection(anchor, ref["anchor"])
+        assert same.mean() > 0.7
+        att = {"out": ref["out"][:, :, None], "lse": ref["lse"][:, :, None]}
+        P.compare_attention(out[:, :, None], lse[:, :, None], att, dtype, where=same[:, :, None])
 
 
 def test_error_returns(sla, handle):
@@ -207,7 +209,12 @@ def test_prefill_host_matches_device_calls(sla, seq_len, dtype):
                                      np.random.default_rng(5).integers(0, seq_len, 200)]))
     hn = P.host_inputs(x)
     code = synth.dtype_code(dtype)
-    ref = O.span_attention(hn["q"], hn["k"], hn["v"], code, np.ascontiguousarray(ha[:, :, rows].numpy()),
-                           span_len=w.span_len, rows=rows)
-    P.compare_attention(ho, hl, ref, dtype, rows=rows)
+    # against the oracle's own search and attention on sampled rows; rows where the two selections
+    # differ (near-ties) are left out of the output comparison
+    ref_s = O.span_search(hn["q_s"], hn["k"], code, top_k=w.top_k, rows=rows)
+    P.compare_search(ha.cuda(), hs.cuda(), ref_s, rows=rows)
+    ref = O.span_attention(hn["q"], hn["k"], hn["v"], code, ref_s["anchor"], span_len=w.span_len, rows=rows)
+    same = P.same_selection(ha[:, :, rows], ref_s["anchor"])
+    assert same.mean() > 0.95
+    P.compare_attention(ho, hl, ref, dtype, rows=rows, where=same)
     handle.close()
