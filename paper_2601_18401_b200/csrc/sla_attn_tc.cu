@@ -2,9 +2,12 @@
 // K/V tiles by TMA, one softmax thread per query row.
 //
 // What it computes is Section "Span attention" (A_{i,t} = Attention(Q(i), K[S_t], V[S_t])) with the
-// spans of Algorithm 1, under union semantics: the k spans of a (query, head) row are sorted and
-// clipped to disjoint "pieces"; every piece is attended on its own and the per-piece results are
-// merged exactly through their log-sum-exp.
+// spans of Algorithm 1.  Union mode: the k spans of a (query, head) row (and its local window) are
+// sorted and clipped to disjoint "pieces"; every piece is attended on its own and the per-piece
+// results are merged exactly through their log-sum-exp.  Per-span mode (Algorithm 1 literally): the
+// pieces are the spans themselves (the part left of the window) plus the window once per row; the
+// merge forms every A_t from its span piece and the window piece and applies the gate of Section
+// "Combination".
 //
 // The systems problem (Section "Kernel design"): neighbouring queries pick different spans, so the
 // rows of one MMA tile must be made to share a key footprint.  Here pieces are grouped by the
@@ -14,15 +17,19 @@
 // shared memory and the tile walks the key blocks they cover from left to right.
 //
 //   tc::prepare          the counting sort and the tile table (sla_attn_prep.cu)
-//   tc_attend            persistent CTAs, tiles handed out through an atomic counter; per tile and
-//                        key block: S = Q K^T (tcgen05, smem x smem -> TMEM), row softmax in
-//                        registers, P (bf16) back into TMEM, O += P V (tcgen05, TMEM x smem -> TMEM)
+//   tc_attend            persistent CTAs, tile t goes to CTA t mod grid (the table is static once
+//                        built); per tile and key block: S = Q K^T (tcgen05, smem x smem -> TMEM), row
+//                        softmax in registers, P (bf16) back into TMEM, O += P V (tcgen05, TMEM x smem
+//                        -> TMEM); per piece a normalised fp16 block-floating-point partial + lse
 //   tc_merge             per row: log-sum-exp merge of its pieces -> out, lse
+//   tc_merge_gated       per row: A_t = merge(span piece, window piece), O = sum_t alpha_t A_t
 //
 // CTA layout of tc_attend (192 threads, two CTAs per SM): warps 0-3 own one tile row each (TMEM lane
-// = row): Q gather, softmax, epilogue; warp 4 issues the MMAs; warp 5 issues the TMA loads.  TMEM:
-// two 64-column S buffers (P aliases the S it came from) and 128 columns of O.  Every wait on an
-// mbarrier is bounded; when one runs out the CTA raises a status bit, drains and leaves.
+// = row): Q gather, softmax, epilogue; one thread of warp 4 issues the MMAs; one thread of warp 5
+// issues the TMA loads (K and V as two independent streams).  TMEM: two 64-column S buffers (P aliases
+// the S it came from) and 128 columns of O.  Every wait on an mbarrier is bounded; when one runs out
+// the CTA raises a status bit, drains and leaves.  The kernel is sensitive to its code size (loops
+// over rarely taken paths stay rolled, the spin loops of the waits are not unrolled).
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <cuda_fp16.h>
