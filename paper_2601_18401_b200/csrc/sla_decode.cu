@@ -54,6 +54,9 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
     const long long i = n_ctx - 1;
     const T *kbase = k + b * c.kv_sb + g * c.kv_sh;
 
+    // the attention kernel of this step may be scheduled now; it waits for this grid to finish before it
+    // touches anything this kernel writes
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     float qv[GT][E];
 #pragma unroll
     for (int t = 0; t < GT; ++t) Vec16<T>::load(q_s + b * c.q_sb + (long long)(h0 + t) * c.q_sh + sub * E, qv[t]);
@@ -230,6 +233,9 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
     const int h = (int)(bh % c.Hq), b = (int)(bh / c.Hq), g = h / c.G;
     const int n_splits = gridDim.x, split = blockIdx.x;
 
+    // launched with programmatic stream serialization: everything above overlaps the tail of the
+    // score kernel, whose results (span table, selected anchors) are read from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int *sp = spans + unit * (2 * pcap + 2);
     const int cnt = sp[2 * pcap + 1];
     for (int j = tid; j < cnt; j += kAttnThreads) s_start[j] = sp[j];
@@ -463,10 +469,20 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
     if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    decode_attn<T, D><<<dim3(p.n_splits, c.B * c.Hq * units), kAttnThreads, 0, st>>>(
-        (const T *)q, kk, (const T *)v, c, spans, partial, done_unit, unit_out, done_head, out_anchor, out_score,
-        (T *)out, lse);
-    return cudaGetLastError();
+    // programmatic dependent launch: the attention grid is set up while the score kernel drains
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.n_splits, c.B * c.Hq * units);
+    cfg.blockDim = dim3(kAttnThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_attn<T, D>, (const T *)q, kk, (const T *)v, c, (const int *)spans, partial,
+                              done_unit, unit_out, done_head, (const int32_t *)out_anchor, (const float *)out_score,
+                              (T *)out, lse);
 }
 
 }  // namespace
