@@ -30,9 +30,12 @@ __device__ __forceinline__ int bucket_of(int lo, int hi, int ncls, int nb_max) {
     return eb * ncls + cls;
 }
 
-template <int PASS>
+// K: compile-time bound on the intervals of a row (anchors + window) for the register-resident piece
+// builder, or 0 for the general one.
+template <int PASS, int K>
 __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
     extern __shared__ int hist[];   // [NB * ncls]
+    constexpr int KA = K > 0 ? K : kMaxTopK + 1;
     const int nk = a.NB * a.ncls;
     const int bg = blockIdx.x / a.ctas_per_bg, part = blockIdx.x % a.ctas_per_bg;
     const int g = bg % a.Hkv, b = bg / a.Hkv;
@@ -43,17 +46,31 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
     int *gcursor = a.key_cursor + (long long)bg * nk;
     for (int x = threadIdx.x; x < nk; x += kPrepThreads) hist[x] = 0;
     __syncthreads();
-
-    int lo[kMaxTopK + 1], hi[kMaxTopK + 1], slot[kMaxTopK + 1];
-    // sub-pass A: this CTA's pieces per bucket
-    for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
+    int lo[KA], hi[KA], slot[KA];
+    auto pieces_of = [&](long long q, int &row) {
         const int hg = (int)((unsigned)q / (unsigned)a.Lc), rc = (int)((unsigned)q % (unsigned)a.Lc);   // G * Lc < 2^31
         const int h = g * a.G + hg;
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
         const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
-        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len, a.len_first, a.n_len), a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
-        if (PASS == 0) a.n_pieces[((long long)b * a.Hq + h) * a.Lc + rc] = (unsigned char)cnt;
-        for (int j = 0; j < cnt; ++j) atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+        row = (int)(((long long)b * a.Hq + h) * a.Lc + rc);
+        const long long ell = base_len(i, a.span_len, a.len_first, a.n_len);
+        if constexpr (K > 0)
+            return row_pieces_small<KA>(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
+        else
+            return row_pieces(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
+    };
+    // sub-pass A: this CTA's pieces per bucket
+    for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
+        int row;
+        const int cnt = pieces_of(q, row);
+        if (PASS == 0) a.n_pieces[row] = (unsigned char)cnt;
+        if constexpr (K > 0) {
+#pragma unroll
+            for (int j = 0; j < KA; ++j)
+                if (j < cnt) atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+        } else {
+            for (int j = 0; j < cnt; ++j) atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+        }
     }
     __syncthreads();
     if constexpr (PASS == 0) {
@@ -68,15 +85,20 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
     __syncthreads();
     // sub-pass B: write the records
     for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
-        const int hg = (int)((unsigned)q / (unsigned)a.Lc), rc = (int)((unsigned)q % (unsigned)a.Lc);   // G * Lc < 2^31
-        const int h = g * a.G + hg;
-        const long long r = a.r0 + rc, i = a.q_pos0 + r;
-        const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
-        const int cnt = row_pieces(an, a.top_k, i, base_len(i, a.span_len, a.len_first, a.n_len), a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
-        const int row = (int)(((long long)b * a.Hq + h) * a.Lc + rc);
-        for (int j = 0; j < cnt; ++j) {
-            const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
-            a.recs[pos] = make_int4(row, slot[j], lo[j], hi[j]);
+        int row;
+        const int cnt = pieces_of(q, row);
+        if constexpr (K > 0) {
+#pragma unroll
+            for (int j = 0; j < KA; ++j)
+                if (j < cnt) {
+                    const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+                    a.recs[pos] = make_int4(row, slot[j], lo[j], hi[j]);
+                }
+        } else {
+            for (int j = 0; j < cnt; ++j) {
+                const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+                a.recs[pos] = make_int4(row, slot[j], lo[j], hi[j]);
+            }
         }
     }
     }
@@ -203,22 +225,27 @@ __global__ void __launch_bounds__(256) prep_tile_bounds(PrepArgs a) {
 cudaError_t prepare(const PrepArgs &a, cudaStream_t st, long long *launches) {
     const int n_bg = a.B * a.Hkv;
     const size_t smem = (size_t)a.NB * a.ncls * sizeof(int);
+    // register-resident piece builder for up to 8 / 16 anchors (+ window), the general one otherwise
+    const int n_iv = a.top_k + (a.window > 0 ? 1 : 0);
+    const int variant = n_iv <= 9 ? 0 : n_iv <= 17 ? 1 : 2;
+    void (*k0)(PrepArgs) = variant == 0 ? prep_pieces<0, 9> : variant == 1 ? prep_pieces<0, 17> : prep_pieces<0, 0>;
+    void (*k1)(PrepArgs) = variant == 0 ? prep_pieces<1, 9> : variant == 1 ? prep_pieces<1, 17> : prep_pieces<1, 0>;
     // function attributes belong to a device's context: remember the largest size set per device
-    static size_t attr_bytes[64] = {};
+    static size_t attr_bytes[64][3] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     const bool known = dev >= 0 && dev < 64;
-    if (smem > 48 * 1024 && (!known || smem > attr_bytes[dev])) {
-        cudaError_t e = cudaFuncSetAttribute(prep_pieces<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(prep_pieces<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (smem > 48 * 1024 && (!known || smem > attr_bytes[dev][variant])) {
+        cudaError_t e = cudaFuncSetAttribute(k0, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        if (known) attr_bytes[dev] = smem;
+        if (known) attr_bytes[dev][variant] = smem;
     }
     const unsigned grid = (unsigned)(n_bg * a.ctas_per_bg);
-    prep_pieces<0><<<grid, kPrepThreads, smem, st>>>(a);
+    k0<<<grid, kPrepThreads, smem, st>>>(a);
     prep_scan_local<<<n_bg, kPrepThreads, 0, st>>>(a);
     prep_scan_global<<<n_bg, kPrepThreads, 0, st>>>(a);
-    prep_pieces<1><<<grid, kPrepThreads, smem, st>>>(a);
+    k1<<<grid, kPrepThreads, smem, st>>>(a);
     prep_tile_bounds<<<(unsigned)((a.max_tiles + 7) / 8), 256, 0, st>>>(a);
     if (launches) *launches += 5;
     return cudaGetLastError();
