@@ -67,6 +67,8 @@ def run_prefill(sla, handle, w, q_pos0=0, Lq=None, permute=False, softmax_scale=
     dict(top_k=1, span_len=100, seq_len=2100),
     dict(back_factor=0, fwd_factor=0, span_len=7),                           # single-token spans
     dict(seq_len=1, top_k=3), dict(seq_len=2, top_k=3), dict(seq_len=5, top_k=2),
+    dict(n_q_heads=16, n_kv_heads=1, seq_len=900, top_k=12, span_len=20),   # widest group, 9..16 anchors per row
+    dict(n_q_heads=12, n_kv_heads=2, seq_len=700, top_k=20, span_len=9),    # group of 6, more than 16 anchors
 ])
 def test_prefill_parity(sla, handle, kw):
     run_prefill(sla, handle, workload(**kw))
