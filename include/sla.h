@@ -231,6 +231,39 @@ sla_status_t sla_decode_step_static(const void *q_s, const void *q, const void *
                                     int64_t n_ctx, const sla_layout_t *layout, const sla_params_t *params,
                                     void *out, float *lse, int32_t *out_anchor, float *out_score, void *stream);
 
+/* ---- sequence-sharded decode step --------------------------------------------------------------
+ *
+ * For a KV cache that is split across devices by position: rank r holds the keys and values of the
+ * contiguous positions [shard_lo, shard_lo + shard_len) of every sequence, as tensors
+ * [B, Hkv, >= shard_len, D] whose index 0 is position shard_lo (kv strides of the layout).  One decode
+ * step is three calls per rank with two small exchanges between them, which the caller carries out
+ * (an all-gather each; the Python package does them with torch.distributed):
+ *
+ *   1. sla_decode_shard_search: scores the anchors of query position n_ctx - 1 that fall into this
+ *      rank's range and returns its top_k best (global positions, -1 / -inf padding)       -> gather
+ *   2. sla_decode_shard_attend: from the candidates of all ranks [n_shards, B, Hq, top_k] picks the
+ *      global top_k (the selection of the unsharded step: larger score first, then the nearer
+ *      anchor), builds their spans (Algorithm 1), attends to the part inside this rank's range and
+ *      returns out_anchor / out_score (the same on every rank) and `partial`
+ *      [B, Hq, D + 2] fp32 = {log-sum-exp, 0, normalised output} of its part                -> gather
+ *   3. sla_decode_shard_merge: merges the partial results of all ranks [n_shards, B, Hq, D + 2]
+ *      through their log-sum-exp into out [B, Hq, D] (input dtype, q strides) and lse [B, Hq].
+ *
+ * The result equals sla_decode_step on the whole cache (Section "Kernel design", "Decoding path").
+ * Union mode without a local window; q_s, q as for sla_decode_step; positions >= n_ctx of a range are
+ * ignored.  All pointers are device memory of this rank. */
+sla_status_t sla_decode_shard_search(sla_handle_t handle, const void *q_s, const void *k_local,
+                                     int64_t shard_lo, int64_t shard_len, int64_t n_ctx,
+                                     const sla_layout_t *layout, const sla_params_t *params,
+                                     int32_t *cand_anchor, float *cand_score, void *stream);
+sla_status_t sla_decode_shard_attend(sla_handle_t handle, const void *q, const void *k_local,
+                                     const void *v_local, int64_t shard_lo, int64_t shard_len, int64_t n_ctx,
+                                     const sla_layout_t *layout, const sla_params_t *params, int32_t n_shards,
+                                     const int32_t *all_anchor, const float *all_score, int32_t *out_anchor,
+                                     float *out_score, float *partial, void *stream);
+sla_status_t sla_decode_shard_merge(sla_handle_t handle, int32_t n_shards, const float *all_partial,
+                                    const sla_layout_t *layout, void *out, float *lse, void *stream);
+
 /* ---- host-buffer convenience calls ---------------------------------------------------------- */
 
 /* sla_span_search followed by sla_span_attention on HOST buffers (pinned memory gives the best

@@ -25,6 +25,7 @@ EXPORTS = [
     "sla_poll_status", "sla_span_search", "sla_span_attention", "sla_decode_step",
     "sla_host_staging_bytes", "sla_prefill_host", "sla_kernel_launches", "sla_set_kernel_timing",
     "sla_kernel_time_ms", "sla_decode_step_static", "sla_span_attention_gated",
+    "sla_decode_shard_search", "sla_decode_shard_attend", "sla_decode_shard_merge",
 ]
 
 
@@ -81,6 +82,12 @@ def load_library():
     lib.sla_span_attention.argtypes = [vp, vp, vp, vp, i64, i64, i64, LP, PP, vp, vp, vp, vp]
     lib.sla_span_attention_gated.restype = i32
     lib.sla_span_attention_gated.argtypes = [vp, vp, vp, vp, i64, i64, i64, LP, PP, vp, vp, vp, vp, vp, vp]
+    lib.sla_decode_shard_search.restype = i32
+    lib.sla_decode_shard_search.argtypes = [vp, vp, vp, i64, i64, i64, LP, PP, vp, vp, vp]
+    lib.sla_decode_shard_attend.restype = i32
+    lib.sla_decode_shard_attend.argtypes = [vp, vp, vp, vp, i64, i64, i64, LP, PP, i32, vp, vp, vp, vp, vp, vp]
+    lib.sla_decode_shard_merge.restype = i32
+    lib.sla_decode_shard_merge.argtypes = [vp, i32, vp, LP, vp, vp, vp]
     lib.sla_decode_step.restype = i32
     lib.sla_decode_step.argtypes = [vp, vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
     lib.sla_decode_step_static.restype = i32
@@ -315,3 +322,55 @@ def sla_prefill_host(handle: Handle, q_s: torch.Tensor, q: torch.Tensor, k: torc
                                       anchor.data_ptr(), score.data_ptr(), _stream_ptr(stream))
     handle.check(rc, "sla_prefill_host")
     return out, lse, anchor, score
+
+
+def sla_decode_shard_search(handle: Handle, q_s: torch.Tensor, k_local: torch.Tensor, shard_lo: int, n_ctx: int,
+                            params: sla_params_t, *, shard_len: Optional[int] = None, stream=None):
+    """q_s [B,Hq,D]; k_local [B,Hkv,>=shard_len,D] holds positions shard_lo.. -> this rank's candidates
+    (anchor int32, score fp32) [B,Hq,k]."""
+    B, Hq, _ = q_s.shape
+    shard_len = k_local.shape[2] if shard_len is None else int(shard_len)
+    anchor = torch.empty(B, Hq, params.top_k, dtype=torch.int32, device=q_s.device)
+    score = torch.empty(B, Hq, params.top_k, dtype=torch.float32, device=q_s.device)
+    layout = make_layout(q_s, k_local, decode=True)
+    rc = handle._lib.sla_decode_shard_search(handle.ptr, q_s.data_ptr(), k_local.data_ptr(), int(shard_lo), shard_len,
+                                             int(n_ctx), C.byref(layout), C.byref(params), anchor.data_ptr(),
+                                             score.data_ptr(), _stream_ptr(stream))
+    handle.check(rc, "sla_decode_shard_search")
+    return anchor, score
+
+
+def sla_decode_shard_attend(handle: Handle, q: torch.Tensor, k_local: torch.Tensor, v_local: torch.Tensor,
+                            shard_lo: int, n_ctx: int, params: sla_params_t, all_anchor: torch.Tensor,
+                            all_score: torch.Tensor, *, shard_len: Optional[int] = None, stream=None):
+    """all_anchor / all_score [n_shards,B,Hq,k] (gathered candidates) -> out_anchor, out_score [B,Hq,k] and
+    this rank's partial result [B,Hq,D+2] fp32."""
+    B, Hq, D = q.shape
+    n_shards = all_anchor.shape[0]
+    assert all_anchor.is_contiguous() and all_score.is_contiguous() and all_anchor.dtype == torch.int32
+    assert all_score.dtype == torch.float32 and all_anchor.shape == (n_shards, B, Hq, params.top_k) == all_score.shape
+    shard_len = k_local.shape[2] if shard_len is None else int(shard_len)
+    out_anchor = torch.empty(B, Hq, params.top_k, dtype=torch.int32, device=q.device)
+    out_score = torch.empty(B, Hq, params.top_k, dtype=torch.float32, device=q.device)
+    partial = torch.empty(B, Hq, D + 2, dtype=torch.float32, device=q.device)
+    layout = make_layout(q, k_local, decode=True)
+    rc = handle._lib.sla_decode_shard_attend(handle.ptr, q.data_ptr(), k_local.data_ptr(), v_local.data_ptr(),
+                                             int(shard_lo), shard_len, int(n_ctx), C.byref(layout), C.byref(params),
+                                             n_shards, all_anchor.data_ptr(), all_score.data_ptr(),
+                                             out_anchor.data_ptr(), out_score.data_ptr(), partial.data_ptr(),
+                                             _stream_ptr(stream))
+    handle.check(rc, "sla_decode_shard_attend")
+    return out_anchor, out_score, partial
+
+
+def sla_decode_shard_merge(handle: Handle, all_partial: torch.Tensor, q_like: torch.Tensor, *, stream=None):
+    """all_partial [n_shards,B,Hq,D+2] fp32 (gathered) -> out [B,Hq,D] (dtype and strides of q_like), lse [B,Hq]."""
+    n_shards, B, Hq, D2 = all_partial.shape
+    assert all_partial.is_contiguous() and all_partial.dtype == torch.float32 and D2 == q_like.shape[-1] + 2
+    out = torch.empty_strided(q_like.shape, q_like.stride(), dtype=q_like.dtype, device=q_like.device)
+    lse = torch.empty(B, Hq, dtype=torch.float32, device=q_like.device)
+    layout = make_layout(q_like, q_like.new_empty(B, 1, 1, q_like.shape[-1]), decode=True)
+    rc = handle._lib.sla_decode_shard_merge(handle.ptr, n_shards, all_partial.data_ptr(), C.byref(layout),
+                                            out.data_ptr(), lse.data_ptr(), _stream_ptr(stream))
+    handle.check(rc, "sla_decode_shard_merge")
+    return out, lse

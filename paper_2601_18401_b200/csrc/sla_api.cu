@@ -137,6 +137,8 @@ sla::Call make_call(const sla_handle_t h, const sla_layout_t *l, const sla_param
     c.status = h ? reinterpret_cast<int *>(h->ws) : nullptr;
     c.off = c.off_host = c.len_first = c.len_first_host = nullptr;
     c.n_off = c.n_len = 0;
+    c.shard_lo = 0;
+    c.shard_hi = Lkv;
     if (h && !is_half(p->search_exponent)) {
         c.off = reinterpret_cast<const int *>(h->ws + kOffTableAt);
         c.off_host = h->off_host.data();
@@ -440,6 +442,97 @@ sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, con
                                        out_score, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_decode_step");
     h->launches += 2;
+    return SLA_OK;
+}
+
+namespace {
+
+// Common checks of the three sequence-sharded calls; fills the call description of this rank.
+sla_status_t shard_call(sla_handle_t h, const sla_layout_t *l, const sla_params_t *p, int64_t n_ctx,
+                        int64_t shard_lo, int64_t shard_len, void *stream, sla::Call *c) {
+    if (const char *why = check_layout_params(l, p, true)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (n_ctx <= 0 || n_ctx > 2147483647LL) return fail(h, SLA_ERR_INVALID_ARG, "n_ctx must be in 1..2^31-1%s");
+    if (shard_lo < 0 || shard_len < 0 || shard_lo + shard_len > 2147483647LL)
+        return fail(h, SLA_ERR_INVALID_ARG, "shard range out of bounds%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (p->window != 0 || p->mode != SLA_UNION)
+        return fail(h, SLA_ERR_UNSUPPORTED, "the sequence-sharded step implements the union mode without a window%s");
+    if (sla_status_t ps = prepare_pattern(h, p, n_ctx, static_cast<cudaStream_t>(stream))) return ps;
+    *c = make_call(h, l, p, 1, n_ctx - 1, n_ctx);
+    c->shard_lo = shard_lo;
+    c->shard_hi = shard_lo + shard_len < n_ctx ? shard_lo + shard_len : n_ctx;   // positions >= n_ctx are not valid yet
+    if (c->shard_hi < c->shard_lo) c->shard_hi = c->shard_lo;
+    if ((size_t)(l->batch) * (l->n_kv_heads + 2 * l->n_q_heads) * sizeof(int) > kCounterEnd - kCounterOffset)
+        return fail(h, SLA_ERR_UNSUPPORTED, "too many (batch, head) pairs for the decode step%s");
+    return SLA_OK;
+}
+
+}  // namespace
+
+sla_status_t sla_decode_shard_search(sla_handle_t h, const void *q_s, const void *k_local, int64_t shard_lo,
+                                     int64_t shard_len, int64_t n_ctx, const sla_layout_t *l,
+                                     const sla_params_t *p, int32_t *cand_anchor, float *cand_score, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (!q_s || !k_local || !cand_anchor || !cand_score) return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
+    if (!aligned16(q_s) || !aligned16(k_local)) return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
+    sla::Call c;
+    if (sla_status_t s = shard_call(h, l, p, n_ctx, shard_lo, shard_len, stream, &c)) return s;
+    // candidate strides of this rank: anchors t = i + 1 - offset with shard_lo <= t < shard_hi
+    const long long i = n_ctx - 1;
+    const int s_first = c.shard_hi > i ? 0 : sla::n_strides(c, i - c.shard_hi);      // offsets <= i + 1 - shard_hi lie right of the range
+    const int s_end = c.shard_lo > i ? 0 : sla::n_strides(c, i - c.shard_lo);        // offsets <= i + 1 - shard_lo reach into it
+    const int n = s_end > s_first ? s_end - s_first : 0;
+    const sla::DecodePlan plan =
+        sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim));
+    if (plan.bytes + kHeaderBytes > h->ws_bytes) return fail(h, SLA_ERR_WORKSPACE, "workspace too small for this decode step%s");
+    if ((size_t)n * sizeof(float) * 8 > 180 * 1024) return fail(h, SLA_ERR_UNSUPPORTED, "context too long for the decode top-k stage%s");
+    cudaError_t e = sla::launch_decode_shard_search(q_s, k_local, c, l->dtype, n_ctx, s_first, n, h->ws + kHeaderBytes,
+                                                    reinterpret_cast<int *>(h->ws + kCounterOffset), cand_anchor,
+                                                    cand_score, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_decode_shard_search");
+    h->launches += 1;
+    return SLA_OK;
+}
+
+sla_status_t sla_decode_shard_attend(sla_handle_t h, const void *q, const void *k_local, const void *v_local,
+                                     int64_t shard_lo, int64_t shard_len, int64_t n_ctx, const sla_layout_t *l,
+                                     const sla_params_t *p, int32_t n_shards, const int32_t *all_anchor,
+                                     const float *all_score, int32_t *out_anchor, float *out_score, float *partial,
+                                     void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (!q || !k_local || !v_local || !all_anchor || !all_score || !out_anchor || !out_score || !partial)
+        return fail(h, SLA_ERR_INVALID_ARG, "NULL tensor pointer%s");
+    if (!aligned16(q) || !aligned16(k_local) || !aligned16(v_local)) return fail(h, SLA_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned%s");
+    if (n_shards < 1 || n_shards > 64) return fail(h, SLA_ERR_INVALID_ARG, "n_shards must be in 1..64%s");
+    sla::Call c;
+    if (sla_status_t s = shard_call(h, l, p, n_ctx, shard_lo, shard_len, stream, &c)) return s;
+    const sla::DecodePlan plan =
+        sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim));
+    if (plan.bytes + kHeaderBytes > h->ws_bytes) return fail(h, SLA_ERR_WORKSPACE, "workspace too small for this decode step%s");
+    cudaError_t e = sla::launch_decode_shard_attend(q, k_local, v_local, c, l->dtype, n_ctx, plan, h->ws + kHeaderBytes,
+                                                    reinterpret_cast<int *>(h->ws + kCounterOffset), n_shards,
+                                                    all_anchor, all_score, out_anchor, out_score, partial,
+                                                    static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_decode_shard_attend");
+    h->launches += 2;
+    return SLA_OK;
+}
+
+sla_status_t sla_decode_shard_merge(sla_handle_t h, int32_t n_shards, const float *all_partial,
+                                    const sla_layout_t *l, void *out, float *lse, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (!l || !all_partial || !out || !lse) return fail(h, SLA_ERR_INVALID_ARG, "NULL pointer%s");
+    if (n_shards < 1 || n_shards > 64) return fail(h, SLA_ERR_INVALID_ARG, "n_shards must be in 1..64%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    if (l->batch <= 0 || l->n_q_heads <= 0 || (l->head_dim != 64 && l->head_dim != 128) ||
+        (l->dtype != SLA_F32 && l->dtype != SLA_BF16) || l->q_stride_b < 0 || l->q_stride_h < l->head_dim)
+        return fail(h, SLA_ERR_INVALID_ARG, "bad layout%s");
+    sla::Call c = {};
+    c.B = l->batch; c.Hq = l->n_q_heads; c.D = l->head_dim;
+    c.q_sb = l->q_stride_b; c.q_sh = l->q_stride_h;
+    cudaError_t e = sla::launch_decode_shard_merge(all_partial, n_shards, c, l->dtype, out, lse, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_decode_shard_merge");
+    h->launches += 1;
     return SLA_OK;
 }
 

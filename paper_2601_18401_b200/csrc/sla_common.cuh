@@ -33,6 +33,8 @@ struct Call {
     int n_off;
     const int *len_first, *len_first_host;
     int n_len;
+    // sequence-sharded decode: the key positions [shard_lo, shard_hi) this rank holds ([0, Lkv) otherwise)
+    long long shard_lo, shard_hi;
 };
 
 // floor(sqrt(x)) for 0 <= x < 2^62, exact.

@@ -119,6 +119,7 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
         topk::select_topk(sc, n, c.top_k, i, cand_v, cand_s, out_anchor + bh * c.top_k, out_score + bh * c.top_k, lane,
                           s_min, c.off);
         __syncwarp();
+        if (!spans) continue;   // sequence-sharded step: the spans are built after the global selection
         // intervals: the spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)])
         // and, last, the local window W = [max(0, i-w+1), i]
         const int n_iv = c.top_k + (c.window > 0 ? 1 : 0);
@@ -213,7 +214,8 @@ __global__ void __launch_bounds__(kAttnThreads)
 decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, Call c,
             const int *__restrict__ spans, float *__restrict__ partial, int *__restrict__ done,
             float *__restrict__ unit_out, int *__restrict__ done_head, const int32_t *__restrict__ sel_anchor,
-            const float *__restrict__ sel_score, T *__restrict__ out, float *__restrict__ lse) {
+            const float *__restrict__ sel_score, T *__restrict__ out, float *__restrict__ lse,
+            float *__restrict__ shard_out) {
     __shared__ int s_last;
     constexpr int E = Vec16<T>::kElems;
     constexpr int LPR = D / E;
@@ -381,8 +383,15 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
     }
     if (!per_span) {
         if (tid < D) {
-            out[b * c.q_sb + (long long)h * c.q_sh + tid] = from_float<T>(o_unit);
-            if (tid == 0) lse[bh] = lse_unit;
+            if (shard_out) {
+                // sequence-sharded step: this rank's share of the head, merged with the others' later
+                float *dst = shard_out + bh * (D + 2);
+                dst[2 + tid] = o_unit;
+                if (tid == 0) { dst[0] = lse_unit; dst[1] = 0.f; }
+            } else {
+                out[b * c.q_sb + (long long)h * c.q_sh + tid] = from_float<T>(o_unit);
+                if (tid == 0) lse[bh] = lse_unit;
+            }
         }
         return;
     }
@@ -482,10 +491,212 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, decode_attn<T, D>, (const T *)q, kk, (const T *)v, c, (const int *)spans, partial,
                               done_unit, unit_out, done_head, (const int32_t *)out_anchor, (const float *)out_score,
-                              (T *)out, lse);
+                              (T *)out, lse, (float *)nullptr);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sequence-sharded decode step (the KV cache of one sequence split into contiguous position ranges, one
+// per rank): every rank scores the anchors that fall into its range and keeps its k best
+// (decode_score without a span table); the candidates of all ranks are gathered; every rank then picks
+// the global k best, clips their spans to its own range (decode_shard_select), attends to that part
+// (decode_attn with a partial result) and, after a second gather, all partial results are merged through
+// their log-sum-exp (decode_shard_merge).  Union mode without a local window.
+
+// One warp per (batch, query head): global top-k of the gathered candidates (larger score first, then the
+// nearer anchor, i.e. the larger position: the order of the unsharded selection) and the table of this
+// rank's pieces: the spans of the selected anchors, sorted, clipped to disjoint pieces and to
+// [shard_lo, shard_hi).
+__global__ void __launch_bounds__(32)
+decode_shard_select(const int32_t *__restrict__ all_anchor, const float *__restrict__ all_score, int n_shards,
+                    Call c, long long n_ctx, long long shard_lo, long long shard_hi, int32_t *__restrict__ out_anchor,
+                    float *__restrict__ out_score, int *__restrict__ spans) {
+    __shared__ int s_lo[kMaxTopK], s_hi[kMaxTopK];
+    const int lane = threadIdx.x;
+    const long long bh = blockIdx.x, n_bh = (long long)c.B * c.Hq;
+    const int k = c.top_k, n = n_shards * k;
+    const long long i = n_ctx - 1;
+    for (int j = lane; j < k; j += 32) {
+        out_anchor[bh * k + j] = -1;
+        out_score[bh * k + j] = -CUDART_INF_F;
+    }
+    __syncwarp();
+    for (int x = lane; x < n; x += 32) {
+        const long long src = ((long long)(x / k) * n_bh + bh) * k + x % k;
+        const int ax = all_anchor[src];
+        if (ax < 0) continue;
+        const uint32_t kx = topk::order_key(all_score[src]);
+        int rank = 0;
+        for (int y = 0; y < n; ++y) {
+            const long long sy = ((long long)(y / k) * n_bh + bh) * k + y % k;
+            const int ay = all_anchor[sy];
+            if (ay < 0) continue;
+            const uint32_t ky = topk::order_key(all_score[sy]);
+            rank += (ky > kx) || (ky == kx && ay > ax);
+        }
+        if (rank < k) {
+            out_anchor[bh * k + rank] = ax;
+            out_score[bh * k + rank] = all_score[src];
+        }
+    }
+    __syncwarp();
+    if (lane == 0) {
+        // spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)]), insertion-sorted
+        const long long ell = base_len(c, i);
+        int m = 0;
+        for (int j = 0; j < k; ++j) {
+            const long long t = out_anchor[bh * k + j];
+            if (t < 0) continue;
+            const long long a = t - (long long)c.back * ell, z = t + (long long)c.fwd * ell;
+            const int l0 = (int)(a > 0 ? a : 0), h0 = (int)(z < i ? z : i);
+            int pos = m;
+            while (pos > 0 && (s_lo[pos - 1] > l0 || (s_lo[pos - 1] == l0 && s_hi[pos - 1] > h0))) {
+                s_lo[pos] = s_lo[pos - 1];
+                s_hi[pos] = s_hi[pos - 1];
+                --pos;
+            }
+            s_lo[pos] = l0;
+            s_hi[pos] = h0;
+            ++m;
+        }
+        const int pcap = k + 1;
+        int *start = spans + bh * (2 * pcap + 2);
+        int *cum = start + pcap;
+        int cnt = 0;
+        long long next_free = 0, total = 0;
+        cum[0] = 0;
+        for (int a = 0; a < m; ++a) {
+            long long j0 = s_lo[a] > next_free ? s_lo[a] : next_free;
+            if ((long long)s_hi[a] + 1 > next_free) next_free = (long long)s_hi[a] + 1;
+            // this rank's part of the piece
+            long long j1 = s_hi[a];
+            if (j0 < shard_lo) j0 = shard_lo;
+            if (j1 > shard_hi - 1) j1 = shard_hi - 1;
+            if (j0 <= j1) {
+                start[cnt] = (int)j0;
+                total += j1 - j0 + 1;
+                cum[cnt + 1] = (int)total;
+                ++cnt;
+            }
+        }
+        start[2 * pcap + 1] = cnt;
+    }
+}
+
+// One CTA per (batch, query head): merge of the ranks' partial results {lse, -, o[D]} (fp32).
+template <typename T, int D>
+__global__ void __launch_bounds__(D)
+decode_shard_merge(const float *__restrict__ all_partial, int n_shards, Call c, T *__restrict__ out,
+                   float *__restrict__ lse) {
+    const long long bh = blockIdx.x, n_bh = (long long)c.B * c.Hq;
+    const int h = (int)(bh % c.Hq), b = (int)(bh / c.Hq), tid = threadIdx.x;
+    float mm = -CUDART_INF_F;
+    for (int w = 0; w < n_shards; ++w) mm = fmaxf(mm, all_partial[((long long)w * n_bh + bh) * (D + 2)]);
+    float den = 0.f, acc = 0.f;
+    if (mm > -CUDART_INF_F) {
+        for (int w = 0; w < n_shards; ++w) {
+            const float *src = all_partial + ((long long)w * n_bh + bh) * (D + 2);
+            if (src[0] == -CUDART_INF_F) continue;
+            const float wt = expf(src[0] - mm);
+            den += wt;
+            acc = fmaf(wt, src[2 + tid], acc);
+        }
+    }
+    out[b * c.q_sb + (long long)h * c.q_sh + tid] = from_float<T>(den > 0.f ? acc / den : 0.f);
+    if (tid == 0) lse[bh] = den > 0.f ? mm + logf(den) : -CUDART_INF_F;
+}
+
+template <typename T, int D>
+cudaError_t shard_search_launch(const void *q_s, const void *k_local, const Call &c, long long n_ctx, int s_first,
+                                int n, void *scratch, int *counters, int32_t *cand_anchor, float *cand_score,
+                                cudaStream_t st) {
+    constexpr int E = Vec16<T>::kElems;
+    constexpr int RPI = 32 / (D / E);
+    float *scores = (float *)scratch;
+    const int rows_per_cta = (kScoreThreads / 32) * RPI * 2;
+    const int gt = c.G % 8 == 0 ? 8 : c.G % 4 == 0 ? 4 : c.G % 2 == 0 ? 2 : 1;
+    dim3 gs(n > 0 ? (n + rows_per_cta - 1) / rows_per_cta : 1, c.B * c.Hkv, c.G / gt);
+    // positions are global: the local slice starts at shard_lo
+    const T *qs = (const T *)q_s, *kk = (const T *)k_local - c.shard_lo * c.kv_st;
+    const size_t smem = (size_t)(kScoreThreads / 32) * (n + 2 * topk::kCap + 4 * (kMaxTopK + 1)) * sizeof(float);
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    cudaError_t e = cudaSuccess;
+#define SLA_LAUNCH_SCORE(GT)                                                                                         \
+    do {                                                                                                             \
+        auto kern = decode_score<T, D, GT>;                                                                          \
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        if (e == cudaSuccess)                                                                                        \
+            kern<<<gs, kScoreThreads, smem, st>>>(qs, kk, c, n_ctx, n, s_first, scores, counters, (int *)nullptr,    \
+                                                  cand_anchor, cand_score);                                         \
+    } while (0)
+    switch (gt) {
+        case 8: SLA_LAUNCH_SCORE(8); break;
+        case 4: SLA_LAUNCH_SCORE(4); break;
+        case 2: SLA_LAUNCH_SCORE(2); break;
+        default: SLA_LAUNCH_SCORE(1); break;
+    }
+#undef SLA_LAUNCH_SCORE
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
+template <typename T, int D>
+cudaError_t shard_attend_launch(const void *q, const void *k_local, const void *v_local, const Call &c, long long n_ctx,
+                                const DecodePlan &p, void *scratch, int *counters, int n_shards,
+                                const int32_t *all_anchor, const float *all_score, int32_t *out_anchor,
+                                float *out_score, float *partial_out, cudaStream_t st) {
+    char *base = (char *)scratch;
+    int *spans = (int *)(base + p.off_spans);
+    float *partial = (float *)(base + p.off_partial);
+    int *done_unit = counters + c.B * c.Hkv, *done_head = done_unit + c.B * c.Hq;
+    decode_shard_select<<<c.B * c.Hq, 32, 0, st>>>(all_anchor, all_score, n_shards, c, n_ctx, c.shard_lo, c.shard_hi,
+                                                   out_anchor, out_score, spans);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const T *kk = (const T *)k_local - c.shard_lo * c.kv_st, *vv = (const T *)v_local - c.shard_lo * c.kv_st;
+    decode_attn<T, D><<<dim3(p.n_splits, c.B * c.Hq), kAttnThreads, 0, st>>>(
+        (const T *)q, kk, vv, c, spans, partial, done_unit, (float *)nullptr, done_head, out_anchor, out_score,
+        (T *)nullptr, (float *)nullptr, partial_out);
+    return cudaGetLastError();
 }
 
 }  // namespace
+
+#define SLA_DISPATCH(fn, ...)                                                                    \
+    (dtype == SLA_F32 ? (c.D == 64 ? fn<float, 64>(__VA_ARGS__) : fn<float, 128>(__VA_ARGS__))   \
+                      : (c.D == 64 ? fn<__nv_bfloat16, 64>(__VA_ARGS__) : fn<__nv_bfloat16, 128>(__VA_ARGS__)))
+
+cudaError_t launch_decode_shard_search(const void *q_s, const void *k_local, const Call &c, int dtype,
+                                       long long n_ctx, int s_first, int n, void *scratch, int *counters,
+                                       int32_t *cand_anchor, float *cand_score, cudaStream_t st) {
+    return SLA_DISPATCH(shard_search_launch, q_s, k_local, c, n_ctx, s_first, n, scratch, counters, cand_anchor,
+                        cand_score, st);
+}
+
+cudaError_t launch_decode_shard_attend(const void *q, const void *k_local, const void *v_local, const Call &c,
+                                       int dtype, long long n_ctx, const DecodePlan &plan, void *scratch,
+                                       int *counters, int n_shards, const int32_t *all_anchor,
+                                       const float *all_score, int32_t *out_anchor, float *out_score,
+                                       float *partial_out, cudaStream_t st) {
+    return SLA_DISPATCH(shard_attend_launch, q, k_local, v_local, c, n_ctx, plan, scratch, counters, n_shards,
+                        all_anchor, all_score, out_anchor, out_score, partial_out, st);
+}
+
+cudaError_t launch_decode_shard_merge(const float *all_partial, int n_shards, const Call &c, int dtype, void *out,
+                                      float *lse, cudaStream_t st) {
+    const unsigned grid = (unsigned)(c.B * c.Hq);
+    if (dtype == SLA_F32) {
+        if (c.D == 64) decode_shard_merge<float, 64><<<grid, 64, 0, st>>>(all_partial, n_shards, c, (float *)out, lse);
+        else decode_shard_merge<float, 128><<<grid, 128, 0, st>>>(all_partial, n_shards, c, (float *)out, lse);
+    } else {
+        if (c.D == 64)
+            decode_shard_merge<__nv_bfloat16, 64><<<grid, 64, 0, st>>>(all_partial, n_shards, c, (__nv_bfloat16 *)out, lse);
+        else
+            decode_shard_merge<__nv_bfloat16, 128><<<grid, 128, 0, st>>>(all_partial, n_shards, c, (__nv_bfloat16 *)out, lse);
+    }
+    return cudaGetLastError();
+}
+#undef SLA_DISPATCH
+
 
 int decode_attn_blocks_per_sm(int dtype, int D) {
     static int cache[2][2] = {{0, 0}, {0, 0}};

@@ -68,6 +68,19 @@ cudaError_t launch_decode(const void *q_s, const void *q, const void *k, const v
                           int dtype, long long n_ctx, const DecodePlan &plan, void *scratch, int *counters,
                           void *out, float *lse, int32_t *out_anchor, float *out_score, cudaStream_t st);
 
+// Sequence-sharded decode step (sla_decode.cu): local candidates of one rank, global selection +
+// attention over this rank's part of the spans, merge of the ranks' partial results.
+cudaError_t launch_decode_shard_search(const void *q_s, const void *k_local, const Call &c, int dtype,
+                                       long long n_ctx, int s_first, int n, void *scratch, int *counters,
+                                       int32_t *cand_anchor, float *cand_score, cudaStream_t st);
+cudaError_t launch_decode_shard_attend(const void *q, const void *k_local, const void *v_local, const Call &c,
+                                       int dtype, long long n_ctx, const DecodePlan &plan, void *scratch,
+                                       int *counters, int n_shards, const int32_t *all_anchor,
+                                       const float *all_score, int32_t *out_anchor, float *out_score,
+                                       float *partial_out, cudaStream_t st);
+cudaError_t launch_decode_shard_merge(const float *all_partial, int n_shards, const Call &c, int dtype, void *out,
+                                      float *lse, cudaStream_t st);
+
 // argument checks of a decode step without a handle (defined in sla_api.cu)
 sla_status_t check_decode_args(const void *q_s, const void *q, const void *k_cache, const void *v_cache,
                                int64_t n_ctx, const sla_layout_t *l, const sla_params_t *p, const void *out,

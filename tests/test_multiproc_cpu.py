@@ -46,3 +46,44 @@ def test_two_ranks_independent_sequences_and_max_timing():
 def test_max_over_ranks_is_identity_without_dist():
     import bench
     assert bench.max_over_ranks(3.5, None, "cpu") == 3.5
+
+
+def _gather_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2601_18401_b200 import sharded
+    # the two exchanges of the sequence-sharded decode step: candidates [B,Hq,k], partial results [B,Hq,D+2]
+    cand = torch.full((2, 3, 4), rank, dtype=torch.int32)
+    part = torch.full((2, 3, 10), float(rank) + 0.5)
+    ga, gp = sharded._gather(cand, None), sharded._gather(part, None)
+    out.put((rank, tuple(ga.shape), ga[:, 0, 0, 0].tolist(), tuple(gp.shape), gp[:, 1, 2, 3].tolist()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_decode_exchanges_two_ranks():
+    """Rank order and shapes of the two all-gathers of the sequence-sharded decode step (gloo, CPU)."""
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 30500 + os.getpid() % 1000
+    procs = [ctx.Process(target=_gather_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, sa, va, sp, vp in res:
+        assert sa == (2, 2, 3, 4) and va == [0, 1]
+        assert sp == (2, 2, 3, 10) and vp == [0.5, 1.5]
+
+
+def test_shard_ranges_tile_the_cache():
+    from paper_2601_18401_b200 import sharded
+    for cap, world in ((1000, 1), (1000, 3), (1048576 + 5, 8), (7, 8), (64, 64)):
+        pos = 0
+        for r in range(world):
+            lo, ln = sharded.shard_range(cap, r, world)
+            assert lo == pos and ln >= 0
+            pos += ln
+        assert pos == cap
