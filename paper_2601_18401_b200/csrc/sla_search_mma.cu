@@ -27,6 +27,7 @@ using bf16 = __nv_bfloat16;
 constexpr int kWarps = 8;
 using topk::kCap;
 using topk::select_topk;
+constexpr int kCand = 2 * 4 * topk::kCapG;   // candidate keys and stride indices: 4 heads x kCapG, or 2 x kCap
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -49,7 +50,7 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
     const int n = n_strides(c, i);
     // Algorithm 1: anchors inside the local window are no candidates; t_s lies in W iff (s+1)^2 <= w
     const int s_min = window_strides(c);
-    float *sc = smem + (size_t)warp * (heads * n_max + 2 * kCap);
+    float *sc = smem + (size_t)warp * (heads * n_max + kCand);
     float *cand_v = sc + heads * n_max;
     int *cand_s = reinterpret_cast<int *>(cand_v + kCap);
 
@@ -96,11 +97,30 @@ search_mma(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, int
         }
     }
     __syncwarp();
+    const int n_cand = n > s_min ? n - s_min : 0;
+    {
+        // all heads of the warp at once, a group of lanes per head, when their number and top_k allow it
+        const long long obase0 = ((((long long)b * c.Hq + g * c.G + head0) * c.Lq) + r) * c.top_k;
+        const long long hstride = c.Lq * c.top_k;
+        uint32_t *ck = reinterpret_cast<uint32_t *>(cand_v);
+        int *cs = reinterpret_cast<int *>(cand_v) + 4 * topk::kCapG;
+        bool done = false;
+        if (heads == 4 && c.top_k <= 8)
+            done = topk::select_topk_grouped<4, 2>(sc, n_max, n_cand, c.top_k, i, ck, cs, out_anchor + obase0,
+                                                   out_score + obase0, hstride, lane, s_min, c.off);
+        else if (heads == 4 && c.top_k <= 16)
+            done = topk::select_topk_grouped<4, 4>(sc, n_max, n_cand, c.top_k, i, ck, cs, out_anchor + obase0,
+                                                   out_score + obase0, hstride, lane, s_min, c.off);
+        else if (heads == 2 && c.top_k <= 16)
+            done = topk::select_topk_grouped<2, 2>(sc, n_max, n_cand, c.top_k, i, ck, cs, out_anchor + obase0,
+                                                   out_score + obase0, hstride, lane, s_min, c.off);
+        if (done) return;
+    }
     for (int hh = 0; hh < heads; ++hh) {
         const int h = g * c.G + head0 + hh;
         const long long obase = ((((long long)b * c.Hq + h) * c.Lq) + r) * c.top_k;
-        select_topk(sc + hh * n_max, n > s_min ? n - s_min : 0, c.top_k, i, cand_v, cand_s, out_anchor + obase,
-                    out_score + obase, lane, s_min, c.off);
+        select_topk(sc + hh * n_max, n_cand, c.top_k, i, cand_v, cand_s, out_anchor + obase, out_score + obase, lane,
+                    s_min, c.off);
     }
 }
 
@@ -110,7 +130,7 @@ bool search_mma_supported(const Call &c, int dtype) {
     if (dtype != SLA_BF16 || c.D != 128 || (long long)c.B * c.Hkv > 65535 || c.kv_st > INT_MAX) return false;
     const int n_max = n_strides(c, c.q_pos0 + c.Lq - 1) + 1;
     const int heads = c.G < 8 ? c.G : 8;
-    return (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float) <= 200 * 1024;
+    return (size_t)kWarps * (heads * n_max + kCand) * sizeof(float) <= 200 * 1024;
 }
 
 cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int32_t *oa, float *os, cudaStream_t st,
@@ -119,7 +139,7 @@ cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int
     const dim3 blocks((unsigned)((c.Lq + kWarps - 1) / kWarps), (unsigned)(c.B * c.Hkv));
     for (int head0 = 0; head0 < c.G; head0 += 8) {
         const int heads = c.G - head0 < 8 ? c.G - head0 : 8;
-        const size_t smem = (size_t)kWarps * (heads * n_max + 2 * kCap) * sizeof(float);
+        const size_t smem = (size_t)kWarps * (heads * n_max + kCand) * sizeof(float);
         if (smem > 48 * 1024) {
             cudaError_t e = cudaFuncSetAttribute(search_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
