@@ -218,7 +218,8 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
             float *__restrict__ shard_out) {
     __shared__ int s_last;
     constexpr int E = Vec16<T>::kElems;
-    constexpr int LPR = D / E;
+    constexpr int C = 2;                  // 16-byte chunks of a token row per lane: chunks sub and sub + LPR
+    constexpr int LPR = D / (E * C);      // lanes per token row
     constexpr int RPI = 32 / LPR;
     constexpr int U = 4;
     constexpr int kWarps = kAttnThreads / 32;
@@ -248,20 +249,25 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
 
     const T *kbase = k + b * c.kv_sb + g * c.kv_sh;
     const T *vbase = v + b * c.kv_sb + g * c.kv_sh;
-    float qv[E];
-    Vec16<T>::load(q + b * c.q_sb + (long long)h * c.q_sh + sub * E, qv);
+    float qv[C][E];
     const float scale2 = c.softmax_scale * kLog2e;
 #pragma unroll
-    for (int e = 0; e < E; ++e) qv[e] *= scale2;
-
-    float m = -CUDART_INF_F, l = 0.f, acc[E];
+    for (int ch = 0; ch < C; ++ch) {
+        Vec16<T>::load(q + b * c.q_sb + (long long)h * c.q_sh + (ch * LPR + sub) * E, qv[ch]);
 #pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+        for (int e = 0; e < E; ++e) qv[ch][e] *= scale2;
+    }
+
+    float m = -CUDART_INF_F, l = 0.f, acc[C][E];
+#pragma unroll
+    for (int ch = 0; ch < C; ++ch)
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[ch][e] = 0.f;
     int piece = 0;
     const int slot = warp * RPI + rsel;
 
     for (long long f0 = f_begin; f0 < f_end; f0 += kSlots * U) {
-        uint4 kraw[U], vraw[U];
+        uint4 kraw[U][C], vraw[U][C];
         bool ok[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -270,26 +276,35 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
             if (ok[u]) {
                 while (f >= s_cum[piece + 1]) ++piece;
                 const long long pos = s_start[piece] + (f - s_cum[piece]);
-                kraw[u] = __ldg(reinterpret_cast<const uint4 *>(kbase + pos * c.kv_st + sub * E));
-                vraw[u] = __ldg(reinterpret_cast<const uint4 *>(vbase + pos * c.kv_st + sub * E));
+#pragma unroll
+                for (int ch = 0; ch < C; ++ch) {
+                    kraw[u][ch] = __ldg(reinterpret_cast<const uint4 *>(kbase + pos * c.kv_st + (ch * LPR + sub) * E));
+                    vraw[u][ch] = __ldg(reinterpret_cast<const uint4 *>(vbase + pos * c.kv_st + (ch * LPR + sub) * E));
+                }
             } else {
-                kraw[u] = make_uint4(0, 0, 0, 0);
-                vraw[u] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int ch = 0; ch < C; ++ch) {
+                    kraw[u][ch] = make_uint4(0, 0, 0, 0);
+                    vraw[u][ch] = make_uint4(0, 0, 0, 0);
+                }
             }
         }
         float x[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            float kv[E];
-            if constexpr (sizeof(T) == 2) {
-                Vec16<__nv_bfloat16>::unpack(kraw[u], kv);
-            } else {
-                kv[0] = __uint_as_float(kraw[u].x); kv[1] = __uint_as_float(kraw[u].y);
-                kv[2] = __uint_as_float(kraw[u].z); kv[3] = __uint_as_float(kraw[u].w);
-            }
             x[u] = 0.f;
 #pragma unroll
-            for (int e = 0; e < E; ++e) x[u] = fmaf(qv[e], kv[e], x[u]);
+            for (int ch = 0; ch < C; ++ch) {
+                float kv[E];
+                if constexpr (sizeof(T) == 2) {
+                    Vec16<__nv_bfloat16>::unpack(kraw[u][ch], kv);
+                } else {
+                    kv[0] = __uint_as_float(kraw[u][ch].x); kv[1] = __uint_as_float(kraw[u][ch].y);
+                    kv[2] = __uint_as_float(kraw[u][ch].z); kv[3] = __uint_as_float(kraw[u][ch].w);
+                }
+#pragma unroll
+                for (int e = 0; e < E; ++e) x[u] = fmaf(qv[ch][e], kv[e], x[u]);
+            }
         }
         float m_new = m;
 #pragma unroll
@@ -300,20 +315,25 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
         const float r = (m == -CUDART_INF_F) ? 0.f : exp2f(m - m_new);
         l *= r;
 #pragma unroll
-        for (int e = 0; e < E; ++e) acc[e] *= r;
+        for (int ch = 0; ch < C; ++ch)
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[ch][e] *= r;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const float p = ok[u] ? exp2f(x[u] - m_new) : 0.f;
             l += p;
-            float vv[E];
-            if constexpr (sizeof(T) == 2) {
-                Vec16<__nv_bfloat16>::unpack(vraw[u], vv);
-            } else {
-                vv[0] = __uint_as_float(vraw[u].x); vv[1] = __uint_as_float(vraw[u].y);
-                vv[2] = __uint_as_float(vraw[u].z); vv[3] = __uint_as_float(vraw[u].w);
-            }
 #pragma unroll
-            for (int e = 0; e < E; ++e) acc[e] = fmaf(p, vv[e], acc[e]);
+            for (int ch = 0; ch < C; ++ch) {
+                float vv[E];
+                if constexpr (sizeof(T) == 2) {
+                    Vec16<__nv_bfloat16>::unpack(vraw[u][ch], vv);
+                } else {
+                    vv[0] = __uint_as_float(vraw[u][ch].x); vv[1] = __uint_as_float(vraw[u][ch].y);
+                    vv[2] = __uint_as_float(vraw[u][ch].z); vv[3] = __uint_as_float(vraw[u][ch].w);
+                }
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[ch][e] = fmaf(p, vv[e], acc[ch][e]);
+            }
         }
         m = m_new;
     }
@@ -328,16 +348,20 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
         const float bb = (om == -CUDART_INF_F) ? 0.f : exp2f(om - mn);
         l = l * a + ol * bb;
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            const float oa = __shfl_xor_sync(0xffffffffu, acc[e], off);
-            acc[e] = acc[e] * a + oa * bb;
-        }
+        for (int ch = 0; ch < C; ++ch)
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const float oa = __shfl_xor_sync(0xffffffffu, acc[ch][e], off);
+                acc[ch][e] = acc[ch][e] * a + oa * bb;
+            }
         m = mn;
     }
     if (rsel == 0) {
         if (sub == 0) { s_m[warp] = m; s_l[warp] = l; }
 #pragma unroll
-        for (int e = 0; e < E; ++e) s_acc[warp][sub * E + e] = acc[e];
+        for (int ch = 0; ch < C; ++ch)
+#pragma unroll
+            for (int e = 0; e < E; ++e) s_acc[warp][(ch * LPR + sub) * E + e] = acc[ch][e];
     }
     __syncthreads();
     if (tid < D) {
