@@ -624,11 +624,10 @@ tc_merge(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
 // attention over the part of S_t left of the window, slot top_k the attention over the window; A_t
 // merges the two through their log-sum-exp, and O = sum_t alpha_t A_t with alpha = softmax of the
 // selected anchors' search scores.  16 threads per row, 8 columns each.
-__device__ __forceinline__ void load_piece(const __half *part_o, const float2 *pl, long long slot, int sub, float w,
-                                           float (&dst)[8]) {
-    const uint32_t eb = (__float_as_uint(pl->y) >> (8 * (sub >> 2))) & 0xffu;
+// dst += w x (eight columns of a piece's block-floating-point output; `exps` holds the chunk exponents)
+__device__ __forceinline__ void add_piece(const uint4 &raw, float exps, int sub, float w, float (&dst)[8]) {
+    const uint32_t eb = (__float_as_uint(exps) >> (8 * (sub >> 2))) & 0xffu;
     const float ws = w * __uint_as_float((eb + 1u) << 23);   // weight x 2^(eb - 126)
-    const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(part_o + slot * kD + sub * 8));
     const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -658,7 +657,11 @@ tc_merge_gated(const __half *__restrict__ part_o, const float2 *__restrict__ par
     const long long ell = base_len(c, i);
     const long long w_lo = i - c.window + 1 > 0 ? i - c.window + 1 : 0;
     const bool has_w = c.window > 0;
-    const float lw = has_w ? pl[c.top_k].x : -CUDART_INF_F;
+    // the window piece is needed by nearly every row: request it with the first loads
+    const float2 pw = has_w ? __ldg(pl + c.top_k) : make_float2(-CUDART_INF_F, 0.f);
+    const uint4 raw_w = has_w ? __ldg(reinterpret_cast<const uint4 *>(part_o + (row * slots + c.top_k) * kD + sub * 8))
+                              : make_uint4(0, 0, 0, 0);
+    const float lw = pw.x;
 
     float smax = -CUDART_INF_F;
     int n_sel = 0;
@@ -722,7 +725,7 @@ tc_merge_gated(const __half *__restrict__ part_o, const float2 *__restrict__ par
             if (lse_span && sub == 0) lse_span[orow * c.top_k + j] = l_t;
         }
     }
-    if (cw != 0.f) load_piece(part_o, pl + c.top_k, row * slots + c.top_k, sub, cw, acc);
+    if (cw != 0.f) add_piece(raw_w, pw.y, sub, cw, acc);
     uint32_t w[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -731,6 +734,141 @@ tc_merge_gated(const __half *__restrict__ part_o, const float2 *__restrict__ par
     }
     *reinterpret_cast<uint4 *>(out + b * c.q_sb + h * c.q_sh + r * c.q_st + sub * 8) = make_uint4(w[0], w[1], w[2], w[3]);
     if (sub == 0) lse[orow] = lse_first;
+}
+
+// The same for top_k <= 8, arranged so that the per-row arithmetic (gate, log-sum-exp weights, base
+// span length) is done once per row: a warp takes 32 consecutive rows; first every lane works out the
+// coefficients of its own row (weight of every span piece, summed weight of the window piece, the
+// log-sum-exps), then the warp walks its rows two at a time, 16 lanes per row and 8 columns per lane,
+// with the coefficients handed over by shuffles.
+constexpr int kGateK = 8;
+__global__ void __launch_bounds__(256)
+tc_merge_gated_rows(const __half *__restrict__ part_o, const float2 *__restrict__ part_lse,
+                    const int32_t *__restrict__ anchor, const float *__restrict__ score, Call c, int slots, int Lc,
+                    long long r0, bf16 *__restrict__ out, float *__restrict__ lse, float *__restrict__ lse_span) {
+    const int lane = threadIdx.x & 31;
+    const long long row0 = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 32;
+    const long long rows = (long long)c.B * c.Hq * Lc;
+    if (row0 >= rows) return;
+    const bool has_w = c.window > 0;
+    // ---- phase A: lane = row
+    float coef[kGateK], cw = 0.f;       // weights of the span pieces and of the window piece
+    uint32_t ex[kGateK], ex_w = 0u;     // their chunk exponents
+    long long out_off = 0;
+#pragma unroll
+    for (int j = 0; j < kGateK; ++j) { coef[j] = 0.f; ex[j] = 0u; }
+    {
+        const long long row = row0 + lane;
+        if (row < rows) {
+            const int rc = (int)((unsigned)row % (unsigned)Lc);   // rows < 2^31
+            const int bh = (int)((unsigned)row / (unsigned)Lc);
+            const int h = bh % c.Hq, b = bh / c.Hq;
+            const long long r = r0 + rc, i = c.q_pos0 + r;
+            const long long orow = ((long long)b * c.Hq + h) * c.Lq + r;
+            out_off = b * c.q_sb + h * c.q_sh + r * c.q_st;
+            const int32_t *an = anchor + orow * c.top_k;
+            const float *sc = score + orow * c.top_k;
+            const float2 *pl = part_lse + row * slots;
+            const long long ell = base_len(c, i);
+            const long long w_lo = i - c.window + 1 > 0 ? i - c.window + 1 : 0;
+            const float2 pw = has_w ? __ldg(pl + c.top_k) : make_float2(-CUDART_INF_F, 0.f);
+            const float lw = pw.x;
+            ex_w = __float_as_uint(pw.y);
+            float scv[kGateK], lj[kGateK];
+            bool sel[kGateK], has_s[kGateK];
+            float smax = -CUDART_INF_F;
+            int n_sel = 0;
+#pragma unroll
+            for (int j = 0; j < kGateK; ++j) {
+                const long long t = j < c.top_k ? an[j] : -1;
+                sel[j] = t >= 0 && t <= i;
+                scv[j] = sel[j] ? sc[j] : -CUDART_INF_F;
+                const long long a = t - (long long)c.back * ell;
+                has_s[j] = sel[j] && (!has_w || (a > 0 ? a : 0) < w_lo);   // a part of S_t lies left of the window
+                const float2 pj = has_s[j] ? __ldg(pl + j) : make_float2(-CUDART_INF_F, 0.f);
+                lj[j] = pj.x;
+                ex[j] = __float_as_uint(pj.y);
+                if (sel[j]) { smax = fmaxf(smax, scv[j]); ++n_sel; }
+            }
+            float sden = 0.f;
+#pragma unroll
+            for (int j = 0; j < kGateK; ++j)
+                if (sel[j]) sden += expf(scv[j] - smax);
+            float lse_first = -CUDART_INF_F;
+            if (n_sel == 0 && has_w) {   // Algorithm 1, empty selection: the window alone
+                cw = 1.f;
+                lse_first = lw * kLn2;
+            }
+            bool first = true;
+#pragma unroll
+            for (int j = 0; j < kGateK; ++j) {
+                if (j >= c.top_k) break;
+                float l_t = -CUDART_INF_F;
+                if (sel[j]) {
+                    const float m = fmaxf(lj[j], lw);
+                    const float wj = has_s[j] ? exp2f(lj[j] - m) : 0.f, ww = has_w ? exp2f(lw - m) : 0.f;
+                    const float den = wj + ww;
+                    const float alpha = expf(scv[j] - smax) / sden;
+                    cw = fmaf(alpha, ww / den, cw);
+                    coef[j] = has_s[j] ? alpha * wj / den : 0.f;
+                    l_t = (m + log2f(den)) * kLn2;
+                    if (first) { lse_first = l_t; first = false; }
+                }
+                if (lse_span) lse_span[orow * c.top_k + j] = l_t;
+            }
+            lse[orow] = lse_first;
+        }
+    }
+    // ---- phase B: two rows per step, 16 lanes per row
+    const int sub = lane & 15, hi = lane >> 4;
+    const int shift = 8 * (sub >> 2);
+#pragma unroll 4
+    for (int rr = 0; rr < 16; ++rr) {
+        const int src = 2 * rr + hi;
+        const long long row = row0 + src;
+        const __half *po = part_o + row * slots * kD + sub * 8;
+        float acc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+        float cf[kGateK + 1];
+        uint32_t ee[kGateK + 1];
+        uint4 raw[kGateK + 1];
+#pragma unroll
+        for (int j = 0; j < kGateK; ++j) {
+            cf[j] = __shfl_sync(0xffffffffu, coef[j], src);
+            ee[j] = __shfl_sync(0xffffffffu, ex[j], src);
+        }
+        cf[kGateK] = __shfl_sync(0xffffffffu, cw, src);
+        ee[kGateK] = __shfl_sync(0xffffffffu, ex_w, src);
+        const long long off = __shfl_sync(0xffffffffu, out_off, src);
+#pragma unroll
+        for (int j = 0; j <= kGateK; ++j) {
+            const int slot = j < kGateK ? j : c.top_k;
+            raw[j] = cf[j] != 0.f ? __ldg(reinterpret_cast<const uint4 *>(po + (long long)slot * kD)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j <= kGateK; ++j)
+            if (cf[j] != 0.f) {
+                const uint32_t eb = (ee[j] >> shift) & 0xffu;
+                const float ws = cf[j] * __uint_as_float((eb + 1u) << 23);   // weight x 2^(eb - 126)
+                const uint32_t rw[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&rw[e]));
+                    acc[2 * e] = fmaf(ws, f.x, acc[2 * e]);
+                    acc[2 * e + 1] = fmaf(ws, f.y, acc[2 * e + 1]);
+                }
+            }
+        if (row < rows) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const __nv_bfloat162 pp = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
+                w[e] = *reinterpret_cast<const uint32_t *>(&pp);
+            }
+            *reinterpret_cast<uint4 *>(out + off + sub * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -894,7 +1032,10 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         tc_attend<<<2 * sm_count, kThreads, kSmemBytes, st>>>(tm_k, tm_v, tp);
         if (timer) timer->end(st);
         const unsigned mblocks = (unsigned)((rows * 16 + 255) / 256);
-        if (c.mode == SLA_PER_SPAN)
+        if (c.mode == SLA_PER_SPAN && c.top_k <= kGateK)
+            tc_merge_gated_rows<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(tp.part_o, tp.part_lse, anchor, score, c,
+                                                                               plan.slots, lc, r0, (bf16 *)out, lse, lse_span);
+        else if (c.mode == SLA_PER_SPAN)
             tc_merge_gated<<<mblocks, 256, 0, st>>>(tp.part_o, tp.part_lse, anchor, score, c, plan.slots, lc, r0,
                                                     (bf16 *)out, lse, lse_span);
         else
