@@ -79,6 +79,8 @@ def run_modes(sla, handle, w, window, q_pos0=0):
     dict(dtype="f32", head_dim=64, n_q_heads=2, n_kv_heads=1, seq_len=700),
     dict(span_len=0, back_factor=4, fwd_factor=2, top_k=2),        # the paper's kernel settings
     dict(top_k=40, seq_len=300, span_len=5),                       # padding; rows with nothing selected
+    dict(top_k=8, span_len=10, seq_len=777),                       # the largest k of the row-parallel gated merge
+    dict(top_k=9, span_len=10, seq_len=777),                       # the smallest k of the general one
 ])
 def test_modes_and_window(sla, handle, kw, window):
     run_modes(sla, handle, workload(**kw), window)
