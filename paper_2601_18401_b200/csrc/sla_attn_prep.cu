@@ -23,11 +23,19 @@ namespace {
 
 constexpr int kPrepThreads = 1024;
 
-__device__ __forceinline__ int bucket_of(int lo, int hi, int ncls, int nb_max) {
-    const int eb = hi / kBK, sb = lo / kBK;
-    int cls = ((eb - sb) * ncls) / nb_max;
-    cls = cls < ncls ? cls : ncls - 1;
-    return eb * ncls + cls;
+// Bucket of a piece: its end block and the class of the number of blocks it covers.  Classes are even
+// steps over [0, nb_single) (a single span) and, for joined pieces, over [nb_single, nb_max).
+__device__ __forceinline__ int bucket_of(int lo, int hi, const PrepArgs &a) {
+    const int eb = hi / kBK, sb = lo / kBK, len = eb - sb;
+    int cls;
+    if (len < a.nb_single || a.ncls == a.ncls1) {
+        cls = (len * a.ncls1) / a.nb_single;
+        cls = cls < a.ncls1 ? cls : a.ncls1 - 1;
+    } else {
+        cls = a.ncls1 + ((len - a.nb_single) * (a.ncls - a.ncls1)) / (a.nb_max - a.nb_single + 1);
+        cls = cls < a.ncls ? cls : a.ncls - 1;
+    }
+    return eb * a.ncls + cls;
 }
 
 // K: compile-time bound on the intervals of a row (anchors + window) for the register-resident piece
@@ -55,9 +63,9 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
         row = (int)(((long long)b * a.Hq + h) * a.Lc + rc);
         const long long ell = base_len(i, a.span_len, a.len_first, a.n_len);
         if constexpr (K > 0)
-            return row_pieces_small<KA>(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
+            return row_pieces_small<KA>(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
         else
-            return row_pieces(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, lo, hi, slot, a.status);
+            return row_pieces(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
     };
     // sub-pass A: this CTA's pieces per bucket
     for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
@@ -67,9 +75,9 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
         if constexpr (K > 0) {
 #pragma unroll
             for (int j = 0; j < KA; ++j)
-                if (j < cnt) atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+                if (j < cnt) atomicAdd(&hist[bucket_of(lo[j], hi[j], a)], 1);
         } else {
-            for (int j = 0; j < cnt; ++j) atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+            for (int j = 0; j < cnt; ++j) atomicAdd(&hist[bucket_of(lo[j], hi[j], a)], 1);
         }
     }
     __syncthreads();
@@ -91,12 +99,12 @@ __global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
 #pragma unroll
             for (int j = 0; j < KA; ++j)
                 if (j < cnt) {
-                    const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+                    const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a)], 1);
                     a.recs[pos] = make_int4(row, slot[j], lo[j], hi[j]);
                 }
         } else {
             for (int j = 0; j < cnt; ++j) {
-                const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a.ncls, a.nb_max)], 1);
+                const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a)], 1);
                 a.recs[pos] = make_int4(row, slot[j], lo[j], hi[j]);
             }
         }

@@ -53,6 +53,7 @@ using tc::kBK;    // keys per block
 using tc::kRows;  // pieces per tile
 constexpr int kThreads = 192;   // 4 row warps, MMA issuer, TMA producer
 constexpr int kTmemCols = 256;
+constexpr int kMaxWalk = 4096;   // most key blocks a tile walks
 constexpr uint32_t kColS = 0;    // S buffers at columns 0 and 64
 constexpr uint32_t kColO = 128;
 constexpr int kQBytes = kRows * kD * 2;      // 32 KiB, two 64-wide halves of 128 rows x 128 B
@@ -928,7 +929,7 @@ bool tc_attention_shape_ok(const Call &c, int dtype) {
     const long long ell = base_len(c, c.q_pos0 + c.Lq - 1);
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     if (c.window > span_tokens) span_tokens = c.window;
-    return span_tokens / kBK + 2 <= 4096;
+    return span_tokens / kBK + 2 <= kMaxWalk;
 }
 
 bool tc_attention_supported(const Call &c, int dtype) {
@@ -945,12 +946,33 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     if (c.window > span_tokens) span_tokens = c.window;   // the window is a piece too
     if (span_tokens > c.Lkv) span_tokens = c.Lkv;
-    p.nb_max = (int)((span_tokens - 1) / kBK + 2);
-    // pieces of a group are ordered by blocks covered, in as many classes as the CTA-local histogram
-    // of the counting sort affords (NB * ncls counters in shared memory)
-    p.ncls = p.nb_max < 8 ? p.nb_max : 8;
-    while (p.ncls > 1 && (size_t)p.NB * p.ncls * 4 > 160 * 1024) p.ncls /= 2;
-    p.ok = (size_t)p.NB * p.ncls * 4 <= 160 * 1024;
+    p.nb_single = (int)((span_tokens - 1) / kBK + 2);
+    // Pieces of a group are ordered by blocks covered, in as many classes as the CTA-local histogram
+    // of the counting sort affords (NB * ncls counters in shared memory): up to 8 for the lengths of a
+    // single span and, in union mode, up to 32 more for pieces joined from spans that overlap or touch.
+    // A tile walks as many key blocks as its longest piece, so pieces are joined only when classes of at
+    // most kJoinWidth blocks reach up to the longest joined piece there can be (all spans and the window
+    // in one); otherwise a few long pieces would make every tile they fall into walk far.
+    const size_t hist_cap = 160 * 1024;
+    constexpr int kJoinWidth = 3;
+    const int ncls_avail = (int)(hist_cap / ((size_t)p.NB * 4));
+    p.ncls1 = p.nb_single < 8 ? p.nb_single : 8;
+    while (p.ncls1 > 1 && p.ncls1 > ncls_avail) p.ncls1 /= 2;
+    int ncls2 = 0;
+    p.nb_max = p.nb_single;
+    if (c.mode == SLA_UNION && ncls_avail > p.ncls1) {
+        long long joined = (long long)c.top_k * ((long long)(c.back + c.fwd) * ell + 1) + c.window;
+        if (joined > c.Lkv) joined = c.Lkv;
+        const long long nb_full = (joined - 1) / kBK + 2, extra = nb_full - p.nb_single;
+        const int avail2 = ncls_avail - p.ncls1 < 32 ? ncls_avail - p.ncls1 : 32;
+        if (extra > 0 && nb_full <= kMaxWalk && extra <= (long long)kJoinWidth * avail2) {
+            ncls2 = (int)(extra < avail2 ? extra : avail2);
+            p.nb_max = (int)nb_full;
+        }
+    }
+    p.merge_cap = ncls2 > 0 ? (p.nb_max - 2) * kBK : 0;   // a piece of T tokens covers at most (T-1)/64 + 2 blocks
+    p.ncls = p.ncls1 + ncls2;
+    p.ok = (size_t)p.NB * p.ncls * 4 <= hist_cap;
     p.ctas_per_bg = (148 + p.n_bg - 1) / p.n_bg;
     const size_t rows = (size_t)c.B * c.Hq * Lc;
     p.slots = c.top_k + (c.window > 0 ? 1 : 0);
@@ -1007,6 +1029,7 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         pa.span_len = c.span_len; pa.back = c.back; pa.fwd = c.fwd; pa.Lq = c.Lq; pa.q_pos0 = c.q_pos0;
         pa.window = c.window; pa.mode = c.mode; pa.len_first = c.len_first; pa.n_len = c.n_len;
         pa.r0 = r0; pa.Lc = lc; pa.NB = plan.NB; pa.nb_max = plan.nb_max; pa.ncls = plan.ncls;
+        pa.nb_single = plan.nb_single; pa.ncls1 = plan.ncls1; pa.merge_cap = plan.merge_cap;
         pa.ctas_per_bg = plan.ctas_per_bg;
         pa.key_count = (int *)(ws + plan.off_key_count);
         pa.key_cursor = (int *)(ws + plan.off_key_cursor);

@@ -25,7 +25,10 @@ struct PrepArgs {
     int Lc;                  // query positions in this chunk
     int NB;                  // 64-key blocks in [0, Lkv)
     int nb_max;              // most blocks a piece can cover
-    int ncls;                // classes of "blocks covered" the pieces are ordered by inside a group
+    int nb_single;           // most blocks a single span (or the window) can cover
+    int ncls;                // classes of "blocks covered" the pieces are ordered by inside a group:
+    int ncls1;               // ncls1 of them divide [0, nb_single), the other ncls - ncls1 divide [nb_single, nb_max)
+    int merge_cap;           // union mode: touching pieces are joined while the result stays within this many tokens
     int ctas_per_bg;         // CTAs that share the rows of one (batch, kv head)
     int *key_count;          // [B*Hkv][NB*ncls]: histogram, then exclusive offsets
     int *key_cursor;         // same shape
@@ -41,14 +44,16 @@ struct PrepArgs {
 // Pieces of one row and the slot each one's partial result goes to (slots per row: top_k, plus one
 // when there is a local window W = [max(0, i-w+1), i]).
 //   union mode     the spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)])
-//                  and W, sorted by (lo, hi) and clipped so that each key is kept once; slots are the
-//                  pieces' ordinals left to right;
+//                  and W, sorted by (lo, hi) and clipped so that each key is kept once; a piece that
+//                  starts right where the one before it ends is joined to it (while the joined piece
+//                  stays within merge_cap tokens): overlapping spans become one longer piece, with one
+//                  partial result; slots are the pieces' ordinals left to right;
 //   per-span mode  J_t = S_t united with W is attended as two disjoint pieces: the part of S_t left of
 //                  W in slot j (the anchor's index in the selection) and W, once per row, in slot top_k.
 // Returns the number of pieces; lo[], hi[], slot[] need top_k + 1 entries.
 __device__ inline int row_pieces(const int32_t *__restrict__ an, int top_k, long long i, long long ell,
-                                 int back, int fwd, int window, int mode, int *lo, int *hi, int *slot,
-                                 int *status) {
+                                 int back, int fwd, int window, int mode, int merge_cap, int *lo, int *hi,
+                                 int *slot, int *status) {
     const int w_lo = (int)(i - window + 1 > 0 ? i - window + 1 : 0);
     int n = 0;
     if (mode == SLA_PER_SPAN) {
@@ -104,10 +109,15 @@ __device__ inline int row_pieces(const int32_t *__restrict__ an, int top_k, long
         const int l0 = lo[a], h0 = hi[a];
         const long long j0 = l0 > next_free ? l0 : next_free;
         if (j0 <= h0) {
-            lo[cnt] = (int)j0;
-            hi[cnt] = h0;
-            slot[cnt] = cnt;
-            ++cnt;
+            // the piece before ends at next_free - 1
+            if (cnt > 0 && j0 == next_free && (long long)h0 - lo[cnt - 1] < merge_cap) {
+                hi[cnt - 1] = h0;
+            } else {
+                lo[cnt] = (int)j0;
+                hi[cnt] = h0;
+                slot[cnt] = cnt;
+                ++cnt;
+            }
         }
         if ((long long)h0 + 1 > next_free) next_free = (long long)h0 + 1;
     }
@@ -119,8 +129,8 @@ __device__ inline int row_pieces(const int32_t *__restrict__ an, int top_k, long
 // nothing is indexed dynamically and the arrays stay in registers.  Same results as row_pieces.
 template <int K>
 __device__ __forceinline__ int row_pieces_small(const int32_t *__restrict__ an, int top_k, long long i, long long ell,
-                                                int back, int fwd, int window, int mode, int (&lo)[K], int (&hi)[K],
-                                                int (&slot)[K], int *status) {
+                                                int back, int fwd, int window, int mode, int merge_cap, int (&lo)[K],
+                                                int (&hi)[K], int (&slot)[K], int *status) {
     const int w_lo = (int)(i - window + 1 > 0 ? i - window + 1 : 0);
     // intervals in slot order; absent ones are (INT_MAX, -1) and sort last
 #pragma unroll
@@ -170,17 +180,22 @@ __device__ __forceinline__ int row_pieces_small(const int32_t *__restrict__ an, 
             lo[x] = l0; lo[x + 1] = l1; hi[x] = h0; hi[x + 1] = h1;
         }
     }
-    int cnt = 0;
+    int cnt = 0, last_lo = 0;   // last_lo: start of the piece written last
     long long next_free = 0;
 #pragma unroll
     for (int a = 0; a < K; ++a) {
         const int l0 = lo[a], h0 = hi[a];
         const long long j0 = l0 > next_free ? l0 : next_free;
         const bool on = h0 >= 0 && j0 <= h0;
+        // the piece before ends at next_free - 1: join a piece that starts right there
+        const bool join = on && cnt > 0 && j0 == next_free && (long long)h0 - last_lo < merge_cap;
 #pragma unroll
-        for (int x = 0; x < K; ++x)
-            if (x <= a && on && x == cnt) { lo[x] = (int)j0; hi[x] = h0; slot[x] = x; }
-        cnt += on;
+        for (int x = 0; x < K; ++x) {
+            if (x <= a && on && !join && x == cnt) { lo[x] = (int)j0; hi[x] = h0; slot[x] = x; }
+            if (x < a && join && x == cnt - 1) hi[x] = h0;
+        }
+        if (on && !join) last_lo = (int)j0;
+        cnt += on && !join;
         if (h0 >= 0 && (long long)h0 + 1 > next_free) next_free = (long long)h0 + 1;
     }
     return cnt;

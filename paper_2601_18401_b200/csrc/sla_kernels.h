@@ -30,7 +30,7 @@ cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int
 // ---- tensor-core span-attention for prefill, bf16 / head_dim 128 (sla_attn_tc.cu) ---------------
 // Scratch layout for one chunk of Lc query positions (all offsets in bytes).
 struct TcPlan {
-    int Lc, n_bg, NB, nb_max, ncls, ctas_per_bg;
+    int Lc, n_bg, NB, nb_max, nb_single, ncls, ncls1, merge_cap, ctas_per_bg;
     int slots;   // partial results per query row: top_k, plus one for the local window
     bool ok;   // false when the shared-memory histogram of the counting sort cannot hold NB buckets
     long long max_tiles;
