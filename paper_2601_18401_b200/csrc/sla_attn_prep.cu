@@ -7,10 +7,10 @@
 // (batch, kv head), counts its pieces in a shared-memory histogram and touches the global counters
 // once per non-empty bucket, so that global atomics stay far below one per piece.
 //
-//   prep_pieces<0>   histogram of bucket sizes (+ number of pieces of every row)
+//   prep_count       the pieces of every row, parked; histogram of bucket sizes; pieces per row
 //   prep_scan_local  per (batch, kv head): exclusive offsets of its buckets, record and tile totals
 //   prep_scan_global per (batch, kv head): global offsets, tile table entries
-//   prep_pieces<1>   piece records to their places
+//   prep_scatter     the parked pieces to their places in the sorted list
 //   prep_tile_bounds per tile: how far back its pieces reach (number of key blocks to walk)
 #include <limits.h>
 
@@ -38,77 +38,115 @@ __device__ __forceinline__ int bucket_of(int lo, int hi, const PrepArgs &a) {
     return eb * a.ncls + cls;
 }
 
+// Rows of one (batch, kv head) are shared out evenly among ctas_per_bg CTAs, the same way in both passes.
+struct Share {
+    int bg, g, b;
+    long long q0, q1;
+};
+__device__ __forceinline__ Share share_of(const PrepArgs &a) {
+    Share s;
+    s.bg = blockIdx.x / a.ctas_per_bg;
+    const int part = blockIdx.x % a.ctas_per_bg;
+    s.g = s.bg % a.Hkv;
+    s.b = s.bg / a.Hkv;
+    const long long rows_bg = (long long)a.G * a.Lc;
+    const long long per = (rows_bg + a.ctas_per_bg - 1) / a.ctas_per_bg;
+    s.q0 = per * part < rows_bg ? per * part : rows_bg;   // a CTA beyond the last row gets an empty range
+    s.q1 = (s.q0 + per < rows_bg) ? s.q0 + per : rows_bg;
+    return s;
+}
+__device__ __forceinline__ int row_of(const PrepArgs &a, const Share &s, long long q, int &h, int &rc) {
+    const int hg = (int)((unsigned)q / (unsigned)a.Lc);   // G * Lc < 2^31
+    rc = (int)((unsigned)q % (unsigned)a.Lc);
+    h = s.g * a.G + hg;
+    return (int)(((long long)s.b * a.Hq + h) * a.Lc + rc);
+}
+
+// Counting pass.  Every piece of the CTA's rows is built once, counted in the CTA's shared-memory
+// histogram (the value the atomic returns is the piece's ordinal within its bucket and CTA) and parked
+// in `stage`; the histogram goes to the global bucket counts and, whole, to cta_hist.
 // K: compile-time bound on the intervals of a row (anchors + window) for the register-resident piece
 // builder, or 0 for the general one.
-template <int PASS, int K>
-__global__ void __launch_bounds__(kPrepThreads) prep_pieces(PrepArgs a) {
+template <int K>
+__global__ void __launch_bounds__(kPrepThreads) prep_count(PrepArgs a) {
     extern __shared__ int hist[];   // [NB * ncls]
     constexpr int KA = K > 0 ? K : kMaxTopK + 1;
     const int nk = a.NB * a.ncls;
-    const int bg = blockIdx.x / a.ctas_per_bg, part = blockIdx.x % a.ctas_per_bg;
-    const int g = bg % a.Hkv, b = bg / a.Hkv;
-    const long long rows_bg = (long long)a.G * a.Lc;
-    const long long per = (rows_bg + a.ctas_per_bg - 1) / a.ctas_per_bg;
-    const long long q0 = per * part, q1 = (q0 + per < rows_bg) ? q0 + per : rows_bg;
-    int *gcount = a.key_count + (long long)bg * nk;
-    int *gcursor = a.key_cursor + (long long)bg * nk;
+    const Share sh = share_of(a);
     for (int x = threadIdx.x; x < nk; x += kPrepThreads) hist[x] = 0;
     __syncthreads();
     int lo[KA], hi[KA], slot[KA];
-    auto pieces_of = [&](long long q, int &row) {
-        const int hg = (int)((unsigned)q / (unsigned)a.Lc), rc = (int)((unsigned)q % (unsigned)a.Lc);   // G * Lc < 2^31
-        const int h = g * a.G + hg;
+    for (long long q = sh.q0 + threadIdx.x; q < sh.q1; q += kPrepThreads) {
+        int h, rc;
+        const int row = row_of(a, sh, q, h, rc);
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
-        const int32_t *an = a.anchor + (((long long)b * a.Hq + h) * a.Lq + r) * a.top_k;
-        row = (int)(((long long)b * a.Hq + h) * a.Lc + rc);
+        const int32_t *an = a.anchor + (((long long)sh.b * a.Hq + h) * a.Lq + r) * a.top_k;
         const long long ell = base_len(i, a.span_len, a.len_first, a.n_len);
+        int cnt;
         if constexpr (K > 0)
-            return row_pieces_small<KA>(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
+            cnt = row_pieces_small<KA>(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
         else
-            return row_pieces(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
-    };
-    // sub-pass A: this CTA's pieces per bucket
-    for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
-        int row;
-        const int cnt = pieces_of(q, row);
-        if (PASS == 0) a.n_pieces[row] = (unsigned char)cnt;
+            cnt = row_pieces(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
+        a.n_pieces[row] = (unsigned char)cnt;
+        int4 *st = a.stage + (long long)row * a.slots;
+        auto park = [&](int j) {
+            const int bucket = bucket_of(lo[j], hi[j], a);
+            const int ord = atomicAdd(&hist[bucket], 1);
+            st[j] = make_int4(lo[j], hi[j], bucket | (slot[j] << 24), ord);
+        };
         if constexpr (K > 0) {
 #pragma unroll
             for (int j = 0; j < KA; ++j)
-                if (j < cnt) atomicAdd(&hist[bucket_of(lo[j], hi[j], a)], 1);
+                if (j < cnt) park(j);
         } else {
-            for (int j = 0; j < cnt; ++j) atomicAdd(&hist[bucket_of(lo[j], hi[j], a)], 1);
+            for (int j = 0; j < cnt; ++j) park(j);
         }
     }
     __syncthreads();
-    if constexpr (PASS == 0) {
-        for (int x = threadIdx.x; x < nk; x += kPrepThreads)
-            if (hist[x]) atomicAdd(gcount + x, hist[x]);
-    } else {
-    // claim a contiguous range of every non-empty bucket for this CTA
+    int *gcount = a.key_count + (long long)sh.bg * nk;
+    int *mine = a.cta_hist + (long long)blockIdx.x * nk;
     for (int x = threadIdx.x; x < nk; x += kPrepThreads) {
-        const int cnt = hist[x];
+        const int c = hist[x];
+        mine[x] = c;
+        if (c) atomicAdd(gcount + x, c);
+    }
+}
+
+// Scatter pass: the CTA claims a contiguous range of every bucket it has pieces in (its count is in
+// cta_hist, the bucket's global offset in key_count by now) and moves its parked pieces to their places.
+__global__ void __launch_bounds__(kPrepThreads) prep_scatter(PrepArgs a) {
+    extern __shared__ int hist[];   // [NB * ncls]: first record of this CTA in every bucket
+    const int nk = a.NB * a.ncls;
+    const Share sh = share_of(a);
+    const int *gcount = a.key_count + (long long)sh.bg * nk;
+    int *gcursor = a.key_cursor + (long long)sh.bg * nk;
+    const int *mine = a.cta_hist + (long long)blockIdx.x * nk;
+    for (int x = threadIdx.x; x < nk; x += kPrepThreads) {
+        const int cnt = mine[x];
         hist[x] = cnt ? gcount[x] + atomicAdd(gcursor + x, cnt) : 0;
     }
     __syncthreads();
-    // sub-pass B: write the records
-    for (long long q = q0 + threadIdx.x; q < q1; q += kPrepThreads) {
-        int row;
-        const int cnt = pieces_of(q, row);
-        if constexpr (K > 0) {
+    // One thread per parked slot, four slots in flight per thread.  The rows of a (batch, kv head) are
+    // consecutive (row = first row + q), so the CTA's slots are one contiguous run of `stage`.
+    const unsigned n_el = (unsigned)((sh.q1 - sh.q0) * a.slots);   // rows x slots < 2^31 for the whole chunk
+    const long long row_base = ((long long)sh.b * a.Hq + sh.g * a.G) * a.Lc + sh.q0;
+    const int4 *st = a.stage + row_base * a.slots;
+    constexpr int U = 4;
+    for (unsigned e0 = threadIdx.x; e0 < n_el; e0 += U * kPrepThreads) {
+        int4 pc[U];
+        int row[U];
+        bool on[U];
 #pragma unroll
-            for (int j = 0; j < KA; ++j)
-                if (j < cnt) {
-                    const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a)], 1);
-                    a.recs[pos] = make_int4(row, slot[j], lo[j], hi[j]);
-                }
-        } else {
-            for (int j = 0; j < cnt; ++j) {
-                const int pos = atomicAdd(&hist[bucket_of(lo[j], hi[j], a)], 1);
-                a.recs[pos] = make_int4(row, slot[j], lo[j], hi[j]);
-            }
+        for (int u = 0; u < U; ++u) {
+            const unsigned e = e0 + u * kPrepThreads;
+            const unsigned ql = e / (unsigned)a.slots, j = e - ql * (unsigned)a.slots;
+            row[u] = (int)(row_base + ql);
+            on[u] = e < n_el && j < a.n_pieces[row[u]];
+            if (on[u]) pc[u] = __ldg(st + e);
         }
-    }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (on[u]) a.recs[hist[pc[u].z & 0xffffff] + pc[u].w] = make_int4(row[u], pc[u].z >> 24, pc[u].x, pc[u].y);
     }
 }
 
@@ -236,18 +274,24 @@ cudaError_t prepare(const PrepArgs &a, cudaStream_t st, long long *launches) {
     // register-resident piece builder for up to 8 / 16 anchors (+ window), the general one otherwise
     const int n_iv = a.top_k + (a.window > 0 ? 1 : 0);
     const int variant = n_iv <= 9 ? 0 : n_iv <= 17 ? 1 : 2;
-    void (*k0)(PrepArgs) = variant == 0 ? prep_pieces<0, 9> : variant == 1 ? prep_pieces<0, 17> : prep_pieces<0, 0>;
-    void (*k1)(PrepArgs) = variant == 0 ? prep_pieces<1, 9> : variant == 1 ? prep_pieces<1, 17> : prep_pieces<1, 0>;
+    void (*k0)(PrepArgs) = variant == 0 ? prep_count<9> : variant == 1 ? prep_count<17> : prep_count<0>;
+    void (*k1)(PrepArgs) = prep_scatter;
     // function attributes belong to a device's context: remember the largest size set per device
-    static size_t attr_bytes[64][3] = {};
+    static size_t attr_bytes[64][4] = {};   // the three counting kernels and the scatter kernel
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     const bool known = dev >= 0 && dev < 64;
-    if (smem > 48 * 1024 && (!known || smem > attr_bytes[dev][variant])) {
-        cudaError_t e = cudaFuncSetAttribute(k0, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        if (known) attr_bytes[dev][variant] = smem;
+    if (smem > 48 * 1024) {
+        if (!known || smem > attr_bytes[dev][variant]) {
+            cudaError_t e = cudaFuncSetAttribute(k0, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            if (known) attr_bytes[dev][variant] = smem;
+        }
+        if (!known || smem > attr_bytes[dev][3]) {
+            cudaError_t e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            if (known) attr_bytes[dev][3] = smem;
+        }
     }
     const unsigned grid = (unsigned)(n_bg * a.ctas_per_bg);
     k0<<<grid, kPrepThreads, smem, st>>>(a);

@@ -966,7 +966,7 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
         const long long nb_full = (joined - 1) / kBK + 2, extra = nb_full - p.nb_single;
         const int avail2 = ncls_avail - p.ncls1 < 32 ? ncls_avail - p.ncls1 : 32;
         if (extra > 0 && nb_full <= kMaxWalk && extra <= (long long)kJoinWidth * avail2) {
-            ncls2 = (int)(extra < avail2 ? extra : avail2);
+            ncls2 = (int)((extra + kJoinWidth - 1) / kJoinWidth);   // fewer classes: fewer global counter updates
             p.nb_max = (int)nb_full;
         }
     }
@@ -983,6 +983,7 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     p.off_counters = off; off = align256(off + 64 + (size_t)p.n_bg * 8);
     p.off_key_count = off; off = align256(off + n_keys * 4);
     p.off_key_cursor = off; off = align256(off + n_keys * 4);
+    p.off_cta_hist = off; off = align256(off + (size_t)p.ctas_per_bg * n_keys * 4);
     p.off_tiles = off; off = align256(off + (size_t)p.max_tiles * 16);
     p.off_recs = off; off = align256(off + slots * 16);
     p.off_npieces = off; off = align256(off + rows);
@@ -1022,7 +1023,7 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
     for (long long r0 = 0; r0 < c.Lq; r0 += Lc) {
         const int lc = (int)((c.Lq - r0 < Lc) ? c.Lq - r0 : Lc);
         const long long rows = (long long)c.B * c.Hq * lc;
-        cudaError_t e = cudaMemsetAsync(ws + plan.off_key_count, 0, plan.off_tiles - plan.off_key_count, st);
+        cudaError_t e = cudaMemsetAsync(ws + plan.off_key_count, 0, plan.off_cta_hist - plan.off_key_count, st);
         if (e != cudaSuccess) return e;
         tc::PrepArgs pa;
         pa.anchor = anchor; pa.B = c.B; pa.Hq = c.Hq; pa.Hkv = c.Hkv; pa.G = c.G; pa.top_k = c.top_k;
@@ -1038,6 +1039,9 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         pa.tiles = (int4 *)(ws + plan.off_tiles);
         pa.max_tiles = (int)plan.max_tiles;
         pa.recs = (int4 *)(ws + plan.off_recs);
+        // the parked pieces borrow the head of the partial-output buffer, which is written only after them
+        pa.stage = (int4 *)(ws + plan.off_part_o); pa.slots = plan.slots;
+        pa.cta_hist = (int *)(ws + plan.off_cta_hist);
         pa.n_pieces = (unsigned char *)(ws + plan.off_npieces);
         pa.status = c.status;
         e = tc::prepare(pa, st, launches);

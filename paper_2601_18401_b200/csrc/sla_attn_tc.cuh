@@ -37,6 +37,10 @@ struct PrepArgs {
     int4 *tiles;
     int max_tiles;
     int4 *recs;
+    int4 *stage;             // [rows][slots] {lo, hi, bucket | slot << 24, ordinal within (CTA, bucket)}: the pieces as
+                             // the counting pass found them, so that the scatter pass need not build them again
+    int slots;               // partial results (and staged pieces) per row
+    int *cta_hist;           // [CTAs][NB*ncls]: every CTA's bucket counts
     unsigned char *n_pieces; // [rows]
     int *status;
 };

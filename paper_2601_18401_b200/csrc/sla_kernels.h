@@ -34,7 +34,7 @@ struct TcPlan {
     int slots;   // partial results per query row: top_k, plus one for the local window
     bool ok;   // false when the shared-memory histogram of the counting sort cannot hold NB buckets
     long long max_tiles;
-    size_t off_counters, off_key_count, off_key_cursor, off_tiles, off_recs, off_npieces, off_part_lse,
+    size_t off_counters, off_key_count, off_key_cursor, off_cta_hist, off_tiles, off_recs, off_npieces, off_part_lse,
         off_part_o, bytes;
 };
 bool tc_attention_shape_ok(const Call &c, int dtype);  // host-only shape test
