@@ -25,8 +25,7 @@ constexpr int kPrepThreads = 1024;
 
 // Bucket of a piece: its end block and the class of the number of blocks it covers.  Classes are even
 // steps over [0, nb_single) (a single span) and, for joined pieces, over [nb_single, nb_max).
-__device__ __forceinline__ int bucket_of(int lo, int hi, const PrepArgs &a) {
-    const int eb = hi / kBK, sb = lo / kBK, len = eb - sb;
+__device__ __forceinline__ int class_of(int len, const PrepArgs &a) {
     int cls;
     if (len < a.nb_single || a.ncls == a.ncls1) {
         cls = (len * a.ncls1) / a.nb_single;
@@ -35,7 +34,79 @@ __device__ __forceinline__ int bucket_of(int lo, int hi, const PrepArgs &a) {
         cls = a.ncls1 + ((len - a.nb_single) * (a.ncls - a.ncls1)) / (a.nb_max - a.nb_single + 1);
         cls = cls < a.ncls ? cls : a.ncls - 1;
     }
-    return eb * a.ncls + cls;
+    return cls;
+}
+__device__ __forceinline__ int bucket_of(int lo, int hi, const PrepArgs &a) {
+    const int eb = hi / kBK, sb = lo / kBK;
+    return eb * a.ncls + class_of(eb - sb, a);
+}
+
+// Union-mode pieces of one row for at most K intervals (anchors + window), streamed: emit(lo, hi, n) is
+// called for the n-th piece, left to right.  Same pieces as row_pieces_small up to the order in which
+// intervals with the same left end are clipped (the union, and with it the attention, is the same).
+// All spans of a row are equally long before clipping, so ordering them by anchor orders them by
+// (lo, hi); the window W = [w_lo, i] takes its place through the anchor that would give lo = w_lo.
+// Keys are 2t for a span and 2t_W + 1 for W (after the spans that start at or before w_lo).
+template <int K, typename Emit>
+__device__ __forceinline__ int union_pieces_stream(const int32_t *__restrict__ an, int top_k, int i, long long ell,
+                                                   int back, int fwd, int window, int merge_cap, int *status,
+                                                   Emit emit) {
+    constexpr unsigned kAbsent = 0xffffffffu;
+    const long long bl64 = (long long)back * ell, fl64 = (long long)fwd * ell;
+    const int bl = bl64 > INT_MAX ? INT_MAX : (int)bl64, fl = fl64 > INT_MAX ? INT_MAX : (int)fl64;
+    const int w_lo = i - window + 1 > 0 ? i - window + 1 : 0;
+    unsigned key[K];
+#pragma unroll
+    for (int j = 0; j < K; ++j) {
+        key[j] = kAbsent;
+        if (j < top_k) {
+            const int t = an[j];
+            if (t > i) atomicOr(status, kStatusBadIndex);
+            else if (t >= 0) key[j] = 2u * (unsigned)t;
+        } else if (j == top_k && window > 0) {
+            unsigned tw = (unsigned)w_lo + (unsigned)bl;
+            if (tw > (unsigned)i + 1u) tw = (unsigned)i + 1u;
+            if (tw > 0x7ffffffeu) tw = 0x7ffffffeu;   // stays below the "absent" key
+            key[j] = 2u * tw + 1u;
+        }
+    }
+#pragma unroll
+    for (int round = 0; round < K; ++round)
+#pragma unroll
+        for (int x = round & 1; x + 1 < K; x += 2) {
+            const unsigned lo_ = min(key[x], key[x + 1]), hi_ = max(key[x], key[x + 1]);
+            key[x] = lo_;
+            key[x + 1] = hi_;
+        }
+    int cnt = 0, cur_lo = 0, cur_hi = -1, next_free = 0;
+    bool have = false;
+#pragma unroll
+    for (int x = 0; x < K; ++x) {
+        const unsigned kx = key[x];
+        const bool present = kx != kAbsent;
+        const int t = (int)(kx >> 1);
+        int l0, h0;
+        if (kx & 1u) {
+            l0 = w_lo;
+            h0 = i;
+        } else {
+            l0 = bl >= t ? 0 : t - bl;
+            h0 = fl >= i - t ? i : t + fl;
+        }
+        const int j0 = l0 > next_free ? l0 : next_free;
+        const bool on = present && j0 <= h0;
+        // the piece in hand ends at next_free - 1: an interval that continues right there is joined to it
+        const bool join = on && have && j0 == next_free && h0 - cur_lo < merge_cap;
+        if (on && !join) {
+            if (have) emit(cur_lo, cur_hi, cnt++);
+            cur_lo = j0;
+            have = true;
+        }
+        if (on) cur_hi = h0;
+        if (present && h0 + 1 > next_free) next_free = h0 + 1;
+    }
+    if (have) emit(cur_lo, cur_hi, cnt++);
+    return cnt;
 }
 
 // Rows of one (batch, kv head) are shared out evenly among ctas_per_bg CTAs, the same way in both passes.
@@ -73,7 +144,10 @@ __global__ void __launch_bounds__(kPrepThreads) prep_count(PrepArgs a) {
     constexpr int KA = K > 0 ? K : kMaxTopK + 1;
     const int nk = a.NB * a.ncls;
     const Share sh = share_of(a);
+    // class of every "blocks covered" value, behind the histogram
+    unsigned char *cls_tbl = reinterpret_cast<unsigned char *>(hist + nk);
     for (int x = threadIdx.x; x < nk; x += kPrepThreads) hist[x] = 0;
+    for (int x = threadIdx.x; x <= a.nb_max; x += kPrepThreads) cls_tbl[x] = (unsigned char)class_of(x, a);
     __syncthreads();
     int lo[KA], hi[KA], slot[KA];
     for (long long q = sh.q0 + threadIdx.x; q < sh.q1; q += kPrepThreads) {
@@ -82,6 +156,20 @@ __global__ void __launch_bounds__(kPrepThreads) prep_count(PrepArgs a) {
         const long long r = a.r0 + rc, i = a.q_pos0 + r;
         const int32_t *an = a.anchor + (((long long)sh.b * a.Hq + h) * a.Lq + r) * a.top_k;
         const long long ell = base_len(i, a.span_len, a.len_first, a.n_len);
+        if constexpr (K > 0) {
+            if (a.mode == SLA_UNION) {
+                int4 *st = a.stage + (long long)row * a.slots;
+                const int n = union_pieces_stream<KA>(an, a.top_k, (int)i, ell, a.back, a.fwd, a.window, a.merge_cap, a.status,
+                                                      [&](int l0, int h0, int ordinal) {
+                                                          const int eb = h0 / kBK, len = eb - l0 / kBK;
+                                                          const int bucket = eb * a.ncls + cls_tbl[len < a.nb_max ? len : a.nb_max];
+                                                          const int ord = atomicAdd(&hist[bucket], 1);
+                                                          st[ordinal] = make_int4(l0, h0, bucket | (ordinal << 24), ord);
+                                                      });
+                a.n_pieces[row] = (unsigned char)n;
+                continue;
+            }
+        }
         int cnt;
         if constexpr (K > 0)
             cnt = row_pieces_small<KA>(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
@@ -121,9 +209,24 @@ __global__ void __launch_bounds__(kPrepThreads) prep_scatter(PrepArgs a) {
     const int *gcount = a.key_count + (long long)sh.bg * nk;
     int *gcursor = a.key_cursor + (long long)sh.bg * nk;
     const int *mine = a.cta_hist + (long long)blockIdx.x * nk;
-    for (int x = threadIdx.x; x < nk; x += kPrepThreads) {
-        const int cnt = mine[x];
-        hist[x] = cnt ? gcount[x] + atomicAdd(gcursor + x, cnt) : 0;
+    // four buckets per thread and round, so that the counts, then the claims, are in flight together
+    for (int x0 = threadIdx.x; x0 < nk; x0 += 4 * kPrepThreads) {
+        int cnt[4], first[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int x = x0 + u * kPrepThreads;
+            cnt[u] = x < nk ? mine[x] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int x = x0 + u * kPrepThreads;
+            first[u] = cnt[u] ? gcount[x] + atomicAdd(gcursor + x, cnt[u]) : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int x = x0 + u * kPrepThreads;
+            if (x < nk) hist[x] = first[u];
+        }
     }
     __syncthreads();
     // One thread per parked slot, four slots in flight per thread.  The rows of a (batch, kv head) are
@@ -134,19 +237,24 @@ __global__ void __launch_bounds__(kPrepThreads) prep_scatter(PrepArgs a) {
     constexpr int U = 4;
     for (unsigned e0 = threadIdx.x; e0 < n_el; e0 += U * kPrepThreads) {
         int4 pc[U];
-        int row[U];
-        bool on[U];
+        int row[U], cnt[U], j[U];
+        // all loads first (a slot beyond the row's count holds stale bytes that are not looked at)
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const unsigned e = e0 + u * kPrepThreads;
-            const unsigned ql = e / (unsigned)a.slots, j = e - ql * (unsigned)a.slots;
+            const unsigned ql = e / (unsigned)a.slots;
+            j[u] = (int)(e - ql * (unsigned)a.slots);
             row[u] = (int)(row_base + ql);
-            on[u] = e < n_el && j < a.n_pieces[row[u]];
-            if (on[u]) pc[u] = __ldg(st + e);
+            cnt[u] = 0;
+            if (e < n_el) {
+                cnt[u] = a.n_pieces[row[u]];
+                pc[u] = __ldg(st + e);
+            }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u)
-            if (on[u]) a.recs[hist[pc[u].z & 0xffffff] + pc[u].w] = make_int4(row[u], pc[u].z >> 24, pc[u].x, pc[u].y);
+            if (j[u] < cnt[u])
+                a.recs[hist[pc[u].z & 0xffffff] + pc[u].w] = make_int4(row[u], pc[u].z >> 24, pc[u].x, pc[u].y);
     }
 }
 
@@ -270,7 +378,8 @@ __global__ void __launch_bounds__(256) prep_tile_bounds(PrepArgs a) {
 
 cudaError_t prepare(const PrepArgs &a, cudaStream_t st, long long *launches) {
     const int n_bg = a.B * a.Hkv;
-    const size_t smem = (size_t)a.NB * a.ncls * sizeof(int);
+    // histogram, and behind it the class table of the counting pass (one byte per length)
+    const size_t smem = (size_t)a.NB * a.ncls * sizeof(int) + (((size_t)a.nb_max + 1 + 15) & ~(size_t)15);
     // register-resident piece builder for up to 8 / 16 anchors (+ window), the general one otherwise
     const int n_iv = a.top_k + (a.window > 0 ? 1 : 0);
     const int variant = n_iv <= 9 ? 0 : n_iv <= 17 ? 1 : 2;

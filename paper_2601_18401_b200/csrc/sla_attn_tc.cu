@@ -973,7 +973,9 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     p.merge_cap = ncls2 > 0 ? (p.nb_max - 2) * kBK : 0;   // a piece of T tokens covers at most (T-1)/64 + 2 blocks
     p.ncls = p.ncls1 + ncls2;
     p.ok = (size_t)p.NB * p.ncls * 4 <= hist_cap;
-    p.ctas_per_bg = (148 + p.n_bg - 1) / p.n_bg;
+    // the work-list kernels hold one CTA per SM (their histogram fills the shared memory): no more CTAs
+    // than SMs, or the last few would run as a second wave
+    p.ctas_per_bg = 148 / p.n_bg > 1 ? 148 / p.n_bg : 1;
     const size_t rows = (size_t)c.B * c.Hq * Lc;
     p.slots = c.top_k + (c.window > 0 ? 1 : 0);
     const size_t slots = rows * p.slots;
