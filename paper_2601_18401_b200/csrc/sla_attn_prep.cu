@@ -9,7 +9,8 @@
 //
 //   prep_count       the pieces of every row, parked; histogram of bucket sizes; pieces per row
 //   prep_scan_local  per (batch, kv head): exclusive offsets of its buckets, record and tile totals
-//   prep_scan_global per (batch, kv head): global offsets, tile table entries
+//   prep_scan_global per (batch, kv head): global offsets, tile table entries (a tile = 128 consecutive
+//                    records of the sorted list, whatever end blocks they fall in)
 //   prep_scatter     the parked pieces to their places in the sorted list
 //   prep_tile_bounds per tile: how far back its pieces reach (number of key blocks to walk)
 #include <limits.h>
@@ -36,9 +37,14 @@ __device__ __forceinline__ int class_of(int len, const PrepArgs &a) {
     }
     return cls;
 }
+// Classes run upwards in even end blocks and downwards in odd ones, so that the sorted list changes
+// length smoothly from one end block to the next (tiles are cut across those boundaries).
+__device__ __forceinline__ int bucket_at(int eb, int cls, const PrepArgs &a) {
+    return eb * a.ncls + ((eb & 1) ? a.ncls - 1 - cls : cls);
+}
 __device__ __forceinline__ int bucket_of(int lo, int hi, const PrepArgs &a) {
     const int eb = hi / kBK, sb = lo / kBK;
-    return eb * a.ncls + class_of(eb - sb, a);
+    return bucket_at(eb, class_of(eb - sb, a), a);
 }
 
 // Union-mode pieces of one row for at most K intervals (anchors + window), streamed: emit(lo, hi, n) is
@@ -162,7 +168,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_count(PrepArgs a) {
                 const int n = union_pieces_stream<KA>(an, a.top_k, (int)i, ell, a.back, a.fwd, a.window, a.merge_cap, a.status,
                                                       [&](int l0, int h0, int ordinal) {
                                                           const int eb = h0 / kBK, len = eb - l0 / kBK;
-                                                          const int bucket = eb * a.ncls + cls_tbl[len < a.nb_max ? len : a.nb_max];
+                                                          const int bucket = bucket_at(eb, cls_tbl[len < a.nb_max ? len : a.nb_max], a);
                                                           const int ord = atomicAdd(&hist[bucket], 1);
                                                           st[ordinal] = make_int4(l0, h0, bucket | (ordinal << 24), ord);
                                                       });
@@ -302,25 +308,15 @@ __global__ void __launch_bounds__(kPrepThreads) prep_scan_local(PrepArgs a) {
         cnt[k] = run;
         run += c;
     }
-    __syncthreads();
-    // tiles: every group (end block) is cut into tiles of kRows records
-    int tiles_local = 0;
-    for (int eb = tid; eb < a.NB; eb += kPrepThreads) {
-        const int first = cnt[eb * a.ncls];
-        const int last = (eb + 1 < a.NB) ? cnt[(eb + 1) * a.ncls] : n_recs;
-        tiles_local += (last - first + kRows - 1) / kRows;
-    }
-    int n_tiles;
-    block_excl_scan(tiles_local, n_tiles, warp_sum);
+    // tiles: the sorted list of the (batch, kv head) is cut every kRows records, across end blocks
     if (tid == 0) {
         a.totals[2 * bg] = n_recs;
-        a.totals[2 * bg + 1] = n_tiles;
+        a.totals[2 * bg + 1] = (n_recs + kRows - 1) / kRows;
     }
 }
 
 // One CTA per (batch, kv head): offsets become global, tile table entries are written.
 __global__ void __launch_bounds__(kPrepThreads) prep_scan_global(PrepArgs a) {
-    __shared__ int warp_sum[32];
     __shared__ int s_base[2];
     const int nk = a.NB * a.ncls, bg = blockIdx.x, tid = threadIdx.x, n_bg = a.B * a.Hkv;
     if (tid == 0) {
@@ -330,47 +326,70 @@ __global__ void __launch_bounds__(kPrepThreads) prep_scan_global(PrepArgs a) {
         s_base[1] = tile_base;
         if (bg == n_bg - 1) {
             const int all = tile_base + a.totals[2 * bg + 1];
-            *a.n_tiles = all < a.max_tiles ? all : a.max_tiles;
+            a.n_tiles[0] = a.n_tiles[1] = all < a.max_tiles ? all : a.max_tiles;   // [1]: the count as cut here
         }
     }
     __syncthreads();
     const int rec_base = s_base[0], tile_base = s_base[1], n_recs = a.totals[2 * bg];
     int *cnt = a.key_count + (long long)bg * nk;
-    // tile entries first (they read the local offsets), in rounds of kPrepThreads groups
-    int carry = 0;
-    for (int eb0 = 0; eb0 < a.NB; eb0 += kPrepThreads) {
-        const int eb = eb0 + tid;
-        int first = 0, n = 0;
-        if (eb < a.NB) {
-            first = cnt[eb * a.ncls];
-            n = ((eb + 1 < a.NB) ? cnt[(eb + 1) * a.ncls] : n_recs) - first;
-        }
-        const int nt = (n + kRows - 1) / kRows;
-        int tot;
-        const int off = block_excl_scan(nt, tot, warp_sum) + carry + tile_base;
-        for (int t = 0; t < nt; ++t) {
-            const int left = n - t * kRows;
-            if (off + t < a.max_tiles)
-                a.tiles[off + t] = make_int4(bg, eb, rec_base + first + t * kRows, left < kRows ? left : kRows);
-        }
-        carry += tot;
+    // tile entries {batch*Hkv + kv head, (end block: filled in by prep_tile_bounds), first record, records}
+    const int nt = (n_recs + kRows - 1) / kRows;
+    for (int t = tid; t < nt; t += kPrepThreads) {
+        const int left = n_recs - t * kRows;
+        if (tile_base + t < a.max_tiles)
+            a.tiles[tile_base + t] = make_int4(bg, 0, rec_base + t * kRows, left < kRows ? left : kRows);
     }
     __syncthreads();
     for (int k = tid; k < nk; k += kPrepThreads) cnt[k] += rec_base;
 }
 
-// One warp per tile: the tile walks the key blocks from the one its furthest-reaching piece starts
-// in up to its end block; the count goes into bits 8.. of the entry's last word.
+// One warp per tile as cut by prep_scan_global (128 consecutive records).  Where two neighbouring
+// records of the tile end more than kGap key blocks apart the tile is split there (the pieces left of
+// the gap would be walked through it for nothing); the extra tiles are appended to the table.  For
+// every tile: the end block of its last piece (second word) and the number of key blocks from the one
+// its furthest-reaching piece starts in up to that end block (bits 8.. of the last word).
+constexpr int kGap = 2;
 __global__ void __launch_bounds__(256) prep_tile_bounds(PrepArgs a) {
-    const int t = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (t >= *a.n_tiles) return;
-    int4 ti = a.tiles[t];
-    int lo = INT_MAX;
-    for (int x = lane; x < ti.w; x += 32) lo = min(lo, a.recs[ti.z + x].z);
-    lo = __reduce_min_sync(0xffffffffu, lo);
-    if (lane == 0) {
-        ti.w |= (ti.y - lo / kBK + 1) << 8;
-        a.tiles[t] = ti;
+    __shared__ int s_eb[8][kRows], s_lo[8][kRows];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * 8 + warp;
+    if (t >= a.n_tiles[1]) return;
+    const int4 ti = a.tiles[t];
+    const int cnt = ti.w;
+    int *eb = s_eb[warp], *lo = s_lo[warp];
+    for (int x = lane; x < cnt; x += 32) {
+        const int4 rec = a.recs[ti.z + x];
+        eb[x] = rec.w / kBK;
+        lo[x] = rec.z;
+    }
+    __syncwarp();
+    int seg0 = 0, n_seg = 0;
+    while (seg0 < cnt) {
+        // first record after seg0 that lies beyond a gap (records are ordered by end block)
+        int seg1 = cnt;
+        for (int x0 = seg0 + 1; x0 < cnt && seg1 == cnt; x0 += 32) {
+            const int x = x0 + lane;
+            const bool cut = x < cnt && eb[x] - eb[x - 1] > kGap;
+            const unsigned m = __ballot_sync(0xffffffffu, cut);
+            if (m) seg1 = x0 + __ffs(m) - 1;
+        }
+        int lo_min = INT_MAX;
+        for (int x = seg0 + lane; x < seg1; x += 32) lo_min = min(lo_min, lo[x]);
+        lo_min = __reduce_min_sync(0xffffffffu, lo_min);
+        const int eb_last = eb[seg1 - 1];
+        int idx = t;
+        if (n_seg > 0) {
+            if (lane == 0) idx = atomicAdd(a.n_tiles, 1);
+            idx = __shfl_sync(0xffffffffu, idx, 0);
+        }
+        if (lane == 0) {
+            if (idx < a.max_tiles)
+                a.tiles[idx] = make_int4(ti.x, eb_last, ti.z + seg0, (seg1 - seg0) | ((eb_last - lo_min / kBK + 1) << 8));
+            else
+                atomicOr(a.status, kStatusBadIndex);   // cannot happen: the table has room for one tile per bucket more
+        }
+        seg0 = seg1;
+        ++n_seg;
     }
 }
 

@@ -13,7 +13,8 @@
 // rows of one MMA tile must be made to share a key footprint.  Here pieces are grouped by the
 // 64-key block their right end falls in (per batch and KV head) and, inside a group, ordered by how
 // many key blocks they cover, with one counting sort (histogram, prefix sum, scatter) -- no
-// comparison sort of the queries.  A tile is 128 pieces of one group: their Q rows are gathered into
+// comparison sort of the queries.  A tile is 128 consecutive pieces of the sorted list (of one group,
+// or of neighbouring groups whose end blocks lie next to each other): their Q rows are gathered into
 // shared memory and the tile walks the key blocks they cover from left to right.
 //
 //   tc::prepare          the counting sort and the tile table (sla_attn_prep.cu)
@@ -980,7 +981,9 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     p.slots = c.top_k + (c.window > 0 ? 1 : 0);
     const size_t slots = rows * p.slots;
     const size_t n_keys = (size_t)p.n_bg * p.NB * p.ncls;
-    p.max_tiles = (long long)(slots / kRows) + (long long)p.n_bg * p.NB + 1;
+    // every (batch, kv head) list is cut every kRows records (one ragged tile each) and split again at
+    // gaps between end blocks (fewer than NB per list)
+    p.max_tiles = (long long)(slots / kRows) + (long long)p.n_bg * (p.NB + 1) + 1;
     size_t off = 0;
     p.off_counters = off; off = align256(off + 64 + (size_t)p.n_bg * 8);
     p.off_key_count = off; off = align256(off + n_keys * 4);

@@ -13,7 +13,8 @@ constexpr int kRows = 128;  // pieces per tile
 // Work list of one chunk of query positions, as laid out in the scratch memory:
 //   recs   int4 {row, slot of the row's partial results, lo, hi}: every piece of every row, ordered by
 //          (batch*Hkv + kv head, 64-key block of hi, class of blocks covered)
-//   tiles  int4 {batch*Hkv + kv head, end block, first record, records | key blocks to walk << 8}
+//   tiles  int4 {batch*Hkv + kv head, end block of the last record, first record, records | key blocks to walk << 8}:
+//          128 consecutive records, split where neighbouring records end more than a few key blocks apart
 //   n_tiles, n_pieces[row], and the per-piece partial results
 struct PrepArgs {
     const int32_t *anchor;   // [B,Hq,Lq,top_k]
