@@ -10,9 +10,10 @@
 // slots in a permuted order (identical for A and B, which leaves the dot product unchanged) so that
 // each lane loads 16 contiguous bytes of a row.
 //
-// Scores go to shared memory; the k best of each head are then selected with warp votes: a
-// threshold from the lanes' maxima, compaction of the candidates above it, and k rounds of a
-// warp-wide arg-max (largest score first, smaller stride index on ties).
+// Scores go to shared memory; the k best of each head are then selected with warp votes, the heads
+// of the warp side by side (a group of lanes per head): a threshold from the lanes' best scores,
+// compaction of the candidates at or above it, and the rank of every candidate among them (largest
+// score first, smaller stride index on ties) as its output slot.
 #include <limits.h>
 #include <math_constants.h>
 
