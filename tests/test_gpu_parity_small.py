@@ -130,6 +130,32 @@ def test_attention_with_foreign_anchors(sla, handle):
     assert sla.sla_poll_status(handle) == sla.SLA_OK
 
 
+@pytest.mark.parametrize("top_k,span_len", [(4, 32), (8, 100), (12, 40)])
+def test_attention_with_clustered_anchors(sla, handle, top_k, span_len):
+    """Anchors of the test's own making, clustered in two far-apart regions (near the query and near the
+    start of the sequence): spans of a row overlap and touch (they are attended as one joined piece), and
+    the sorted work list has long runs of key blocks in which no piece ends (tiles are cut there)."""
+    from paper_2601_18401_b200 import synth
+    L = 6000
+    w = workload(seq_len=L, span_len=span_len, top_k=top_k)
+    x = synth.make_prefill(w, device="cuda:0")
+    g = torch.Generator().manual_seed(11)
+    i = torch.arange(L)[None, None, :, None]
+    near = i - (torch.rand(1, 4, L, top_k, generator=g) * 3 * span_len).long()       # overlapping spans next to i
+    far = (torch.rand(1, 4, L, top_k, generator=g) * 200).long()                       # all of them in the first 200 keys
+    pick_far = torch.rand(1, 4, L, top_k, generator=g) < 0.4
+    anchor = torch.where(pick_far, far, near).clamp(min=0)
+    anchor = torch.minimum(anchor, i.expand_as(anchor))
+    anchor[..., top_k - 1] = torch.where(torch.rand(1, 4, L, generator=g) < 0.2, torch.full((1, 4, L), -1), anchor[..., top_k - 1])
+    anchor = anchor.to(torch.int32).cuda()
+    params = sla.make_params(top_k, span_len, head_dim=128)
+    out, lse = sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params)
+    torch.cuda.synchronize()
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    ref = P.oracle_attention_for(P.host_inputs(x), O.BF16, anchor.cpu().numpy(), w)   # the test's own anchors
+    P.compare_attention(out, lse, ref, "bf16")
+
+
 @pytest.mark.parametrize("dtype,D,Hq,Hkv", [("bf16", 128, 8, 2), ("f32", 64, 2, 2), ("bf16", 64, 4, 1), ("f32", 128, 3, 1)])
 def test_decode_parity(sla, handle, dtype, D, Hq, Hkv):
     from paper_2601_18401_b200 import synth
