@@ -48,7 +48,7 @@ __device__ __forceinline__ int bucket_of(int lo, int hi, const PrepArgs &a) {
 }
 
 // Union-mode pieces of one row for at most K intervals (anchors + window), streamed: emit(lo, hi, n) is
-// called for the n-th piece, left to right.  Same pieces as row_pieces_small up to the order in which
+// called for the n-th piece, left to right.  Same pieces as row_pieces up to the order in which
 // intervals with the same left end are clipped (the union, and with it the attention, is the same).
 // All spans of a row are equally long before clipping, so ordering them by anchor orders them by
 // (lo, hi); the window W = [w_lo, i] takes its place through the anchor that would give lo = w_lo.
@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_count(PrepArgs a) {
         }
         int cnt;
         if constexpr (K > 0)
-            cnt = row_pieces_small<KA>(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
+            cnt = row_pieces_per_span_small<KA>(an, a.top_k, i, ell, a.back, a.fwd, a.window, lo, hi, slot, a.status);
         else
             cnt = row_pieces(an, a.top_k, i, ell, a.back, a.fwd, a.window, a.mode, a.merge_cap, lo, hi, slot, a.status);
         a.n_pieces[row] = (unsigned char)cnt;

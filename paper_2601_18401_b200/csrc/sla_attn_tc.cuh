@@ -129,15 +129,16 @@ __device__ inline int row_pieces(const int32_t *__restrict__ an, int top_k, long
     return cnt;
 }
 
-// Register-resident form of row_pieces for at most K - 1 anchors (K intervals with the window): the
-// intervals are sorted with a fixed odd-even transposition network and every loop is unrolled, so that
-// nothing is indexed dynamically and the arrays stay in registers.  Same results as row_pieces.
+// Register-resident form of row_pieces in the per-span mode for at most K - 1 anchors (K intervals with
+// the window): every loop is unrolled and nothing is indexed dynamically, so the arrays stay in
+// registers.  Same results as row_pieces.  (The union mode has its own streaming builder next to the
+// kernel that uses it.)
 template <int K>
-__device__ __forceinline__ int row_pieces_small(const int32_t *__restrict__ an, int top_k, long long i, long long ell,
-                                                int back, int fwd, int window, int mode, int merge_cap, int (&lo)[K],
-                                                int (&hi)[K], int (&slot)[K], int *status) {
+__device__ __forceinline__ int row_pieces_per_span_small(const int32_t *__restrict__ an, int top_k, long long i,
+                                                         long long ell, int back, int fwd, int window, int (&lo)[K],
+                                                         int (&hi)[K], int (&slot)[K], int *status) {
     const int w_lo = (int)(i - window + 1 > 0 ? i - window + 1 : 0);
-    // intervals in slot order; absent ones are (INT_MAX, -1) and sort last
+    // intervals in slot order; absent ones are (INT_MAX, -1)
 #pragma unroll
     for (int j = 0; j < K; ++j) {
         int l0 = INT_MAX, h0 = -1;
@@ -149,7 +150,7 @@ __device__ __forceinline__ int row_pieces_small(const int32_t *__restrict__ an, 
                 const long long a = t - (long long)back * ell, z = t + (long long)fwd * ell;
                 l0 = (int)(a > 0 ? a : 0);
                 h0 = (int)(z < i ? z : i);
-                if (mode == SLA_PER_SPAN && window > 0 && h0 >= w_lo) h0 = w_lo - 1;
+                if (window > 0 && h0 >= w_lo) h0 = w_lo - 1;
                 if (l0 > h0) { l0 = INT_MAX; h0 = -1; }
             }
         } else if (j == top_k && window > 0) {
@@ -160,48 +161,16 @@ __device__ __forceinline__ int row_pieces_small(const int32_t *__restrict__ an, 
         hi[j] = h0;
         slot[j] = j;
     }
-    if (mode == SLA_PER_SPAN) {
-        // pieces keep their slots; compact the present ones to the front, in order
-        int cnt = 0;
+    // pieces keep their slots; compact the present ones to the front, in order
+    int cnt = 0;
 #pragma unroll
-        for (int j = 0; j < K; ++j) {
-            const bool on = hi[j] >= 0;
-            const int l0 = lo[j], h0 = hi[j];
+    for (int j = 0; j < K; ++j) {
+        const bool on = hi[j] >= 0;
+        const int l0 = lo[j], h0 = hi[j];
 #pragma unroll
-            for (int x = 0; x < K; ++x)
-                if (x <= j && on && x == cnt) { lo[x] = l0; hi[x] = h0; slot[x] = j; }
-            cnt += on;
-        }
-        return cnt;
-    }
-    // union mode: sort by (lo, hi), clip to disjoint pieces
-#pragma unroll
-    for (int round = 0; round < K; ++round) {
-#pragma unroll
-        for (int x = round & 1; x + 1 < K; x += 2) {
-            const bool swap = lo[x] > lo[x + 1] || (lo[x] == lo[x + 1] && hi[x] > hi[x + 1]);
-            const int l0 = swap ? lo[x + 1] : lo[x], l1 = swap ? lo[x] : lo[x + 1];
-            const int h0 = swap ? hi[x + 1] : hi[x], h1 = swap ? hi[x] : hi[x + 1];
-            lo[x] = l0; lo[x + 1] = l1; hi[x] = h0; hi[x + 1] = h1;
-        }
-    }
-    int cnt = 0, last_lo = 0;   // last_lo: start of the piece written last
-    long long next_free = 0;
-#pragma unroll
-    for (int a = 0; a < K; ++a) {
-        const int l0 = lo[a], h0 = hi[a];
-        const long long j0 = l0 > next_free ? l0 : next_free;
-        const bool on = h0 >= 0 && j0 <= h0;
-        // the piece before ends at next_free - 1: join a piece that starts right there
-        const bool join = on && cnt > 0 && j0 == next_free && (long long)h0 - last_lo < merge_cap;
-#pragma unroll
-        for (int x = 0; x < K; ++x) {
-            if (x <= a && on && !join && x == cnt) { lo[x] = (int)j0; hi[x] = h0; slot[x] = x; }
-            if (x < a && join && x == cnt - 1) hi[x] = h0;
-        }
-        if (on && !join) last_lo = (int)j0;
-        cnt += on && !join;
-        if (h0 >= 0 && (long long)h0 + 1 > next_free) next_free = (long long)h0 + 1;
+        for (int x = 0; x < K; ++x)
+            if (x <= j && on && x == cnt) { lo[x] = l0; hi[x] = h0; slot[x] = j; }
+        cnt += on;
     }
     return cnt;
 }
