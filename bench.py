@@ -38,9 +38,9 @@ METRIC = "prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one tc_attend launch of the default workload
 # (L = 65536), from the one-pass ncu capture of the full-size launch summarised in profiles/
-TC_ATTEND_DRAM_BYTES_PER_LAUNCH = {65536: 4.73e9, 16384: 0.835e9}
+TC_ATTEND_DRAM_BYTES_PER_LAUNCH = {65536: 4.74e9, 16384: 0.887e9}
 # the same for one decode_attn launch (the dominant kernel of a decode step), by workload
-DECODE_ATTN_DRAM_BYTES_PER_LAUNCH = {"decode_1M": 485.7e6, "decode_10M": 1570.8e6}
+DECODE_ATTN_DRAM_BYTES_PER_LAUNCH = {"decode_1M": 485.2e6, "decode_10M": 1571.4e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
