@@ -951,9 +951,11 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     // Pieces of a group are ordered by blocks covered, in as many classes as the CTA-local histogram
     // of the counting sort affords (NB * ncls counters in shared memory): up to 8 for the lengths of a
     // single span and, in union mode, up to 32 more for pieces joined from spans that overlap or touch.
-    // A tile walks as many key blocks as its longest piece, so pieces are joined only when classes of at
-    // most kJoinWidth blocks reach up to the longest joined piece there can be (all spans and the window
-    // in one); otherwise a few long pieces would make every tile they fall into walk far.
+    // A tile walks as many key blocks as its longest piece, so a joined piece may only be as long as the
+    // classes can still tell apart: when classes of at most kJoinWidth blocks reach up to the longest
+    // joined piece there can be (all spans and the window in one), everything that touches is joined;
+    // otherwise the classes are shared between single spans and joined pairs, and a piece stops growing
+    // at twice a span (measured on the 262144-token configuration: pairs -4 %, triples +1 %).
     const size_t hist_cap = 160 * 1024;
     constexpr int kJoinWidth = 3;
     const int ncls_avail = (int)(hist_cap / ((size_t)p.NB * 4));
@@ -964,11 +966,19 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     if (c.mode == SLA_UNION && ncls_avail > p.ncls1) {
         long long joined = (long long)c.top_k * ((long long)(c.back + c.fwd) * ell + 1) + c.window;
         if (joined > c.Lkv) joined = c.Lkv;
-        const long long nb_full = (joined - 1) / kBK + 2, extra = nb_full - p.nb_single;
+        long long nb_full = (joined - 1) / kBK + 2;
+        if (nb_full > kMaxWalk) nb_full = kMaxWalk;
+        const long long extra = nb_full - p.nb_single;
         const int avail2 = ncls_avail - p.ncls1 < 32 ? ncls_avail - p.ncls1 : 32;
-        if (extra > 0 && nb_full <= kMaxWalk && extra <= (long long)kJoinWidth * avail2) {
+        if (extra > 0 && extra <= (long long)kJoinWidth * avail2) {
             ncls2 = (int)((extra + kJoinWidth - 1) / kJoinWidth);   // fewer classes: fewer global counter updates
             p.nb_max = (int)nb_full;
+        } else if (extra > 0 && ncls_avail >= 4) {
+            if (p.ncls1 > ncls_avail / 2) p.ncls1 = ncls_avail / 2;
+            const int want2 = (p.nb_single + kJoinWidth - 1) / kJoinWidth;
+            ncls2 = ncls_avail - p.ncls1 < want2 ? ncls_avail - p.ncls1 : want2;
+            if (ncls2 > 32) ncls2 = 32;
+            p.nb_max = 2LL * p.nb_single < nb_full ? 2 * p.nb_single : (int)nb_full;
         }
     }
     p.merge_cap = ncls2 > 0 ? (p.nb_max - 2) * kBK : 0;   // a piece of T tokens covers at most (T-1)/64 + 2 blocks
