@@ -36,9 +36,6 @@
 #include <cuda_fp16.h>
 #include <limits.h>
 #include <math_constants.h>
-#ifdef SLA_TC_TIMING
-#include <stdio.h>
-#endif
 
 #include "sla_attn_tc.cuh"
 #include "sla_tc_ptx.cuh"
@@ -130,9 +127,6 @@ __device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) 
     return desc;
 }
 __device__ __forceinline__ float ex2_approx(float x) {
-#ifdef SLA_EXP_NOMUFU
-    return fmaf(x, 1e-3f, 1.f);
-#endif
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
