@@ -12,7 +12,8 @@
 //   prep_scan_global per (batch, kv head): global offsets, tile table entries (a tile = 128 consecutive
 //                    records of the sorted list, whatever end blocks they fall in)
 //   prep_scatter     the parked pieces to their places in the sorted list
-//   prep_tile_bounds per tile: how far back its pieces reach (number of key blocks to walk)
+//   prep_tile_bounds per tile: split where neighbouring pieces end far apart; the tile's end block and how
+//                    far back its pieces reach (number of key blocks to walk)
 #include <limits.h>
 
 #include "sla_attn_tc.cuh"
