@@ -37,7 +37,15 @@
  * (a cudaStream_t passed as void*; NULL = the default stream) and outputs are valid once the stream
  * reaches that point.  The library allocates device memory only in sla_create (the workspace);
  * no call allocates per invocation.  One handle must not be used by two streams at the same time
- * (the workspace is shared).
+ * (the workspace is shared); calls that follow each other on different streams are fine as far as the
+ * library's own tables go (it orders them itself), the caller orders the tensors.
+ *
+ * Kernels: bf16 tensors with head_dim 128 whose K/V dimensions nest in memory (no broadcast views)
+ * run on the tensor-core kernels (span-attention) and the register-MMA kernel (span-search); every
+ * other supported layout -- fp32, head_dim 64, a stride-0 K/V dimension, a single call over more than
+ * about 2.6 million keys -- runs on generic fp32-accumulating kernels with the same results and far
+ * lower throughput.  The choice depends on shapes and strides alone, never on the workspace size: a
+ * workspace too small for the chosen kernel is SLA_ERR_WORKSPACE.
  *
  * Errors: every call returns an sla_status_t; 0 is success, negative values are errors.  When
  * argument validation fails nothing is launched.  No exception or abort crosses this interface.
@@ -140,6 +148,17 @@ int64_t sla_kernel_launches(sla_handle_t handle);
 sla_status_t sla_set_kernel_timing(sla_handle_t handle, int enable);
 sla_status_t sla_kernel_time_ms(sla_handle_t handle, float *ms, int32_t *n_launches);
 
+/* The two integer tables the library derives from exponents other than 1/2 (host-only diagnostics, so
+ * that the rounding rule stated at sla_params_t can be checked without a device; Section "Span
+ * attention", anchors at i - (s+1)^(1/p) + 1, and l(i) proportional to i^p):
+ *   sla_pattern_offsets    out[s] = ceil((s+1)^(1/search_exponent)) for every stride with out[s] <= reach
+ *   sla_pattern_len_steps  out[v-1] = smallest i >= 1 with ceil(i^span_exponent) >= v, for every v
+ *                          reached by some i <= reach
+ * Both return the number of entries (only the first `cap` are written; out may be NULL when cap = 0),
+ * or -1 for an exponent outside [0.2, 0.8] or more than 65536 entries. */
+int32_t sla_pattern_offsets(double search_exponent, int64_t reach, int32_t *out, int32_t cap);
+int32_t sla_pattern_len_steps(double span_exponent, int64_t reach, int32_t *out, int32_t cap);
+
 /* ---- span-search (Section "Span search"; Algorithm 1 scoring and TopK lines) -------------- */
 
 /* Query row r (0 <= r < Lq) is position i = q_pos0 + r; keys 0 .. Lkv-1 are valid; requires
@@ -213,13 +232,19 @@ sla_status_t sla_decode_step(sla_handle_t handle, const void *q_s, const void *q
  *
  * Arguments, results and launch behaviour are those of sla_decode_step (same kernels); inputs and
  * outputs are still the caller's device buffers.  Differences:
- *   - only the union mode without a local window (params->window = 0, params->mode = SLA_UNION);
- *     anything else returns SLA_ERR_UNSUPPORTED;
+ *   - only the union mode without a local window and with the exponents of the quadratic pattern
+ *     (params->window = 0, params->mode = SLA_UNION, search_exponent and span_exponent 0 or 0.5: other
+ *     exponents need tables that live in a handle's workspace); anything else returns
+ *     SLA_ERR_UNSUPPORTED;
  *   - a step whose scratch exceeds the fixed array (it grows with batch * heads * sqrt(n_ctx) and
  *     with batch * heads * splits) is rejected with SLA_ERR_WORKSPACE and nothing is launched; the
  *     1M- and 10M-token configurations with 32 query heads need well under 1 MiB;
- *   - the first call on a device resolves the array's device address (once per device, with that
- *     device current) and asks a few device attributes; make this first call outside any stream
+ *   - set-up happens inside the call, not at load time: the first call on a device resolves the
+ *     array's device address (once per device, with that device current); the first call for each
+ *     (device, dtype, head_dim) asks the device for its SM count and the kernel's occupancy; and the
+ *     first call on a device whose context is long enough for the scoring kernel to need more than
+ *     48 KiB of shared memory (beyond about 1.3 million tokens) raises that kernel's limit, once.  Make
+ *     one call per (device, dtype, head_dim), at the longest context you will use, before any stream
  *     capture;
  *   - all calls on one device share the array: it keeps the previous call's contents (the part that
  *     must start at zero is cleared on the stream at the start of each call), and two calls that

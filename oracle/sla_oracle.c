@@ -20,8 +20,7 @@
  *     scores, O_i = sum_t alpha_t A_{i,t}.
  *   - Sliding window W and DedupConcat, Algorithm 1 lines for W, T = Anchors(i) \ W and J_t.
  *
- * Readings taken where the paper is silent or inconsistent (all are conventions, listed again in
- * the design notes of the repository):
+ * Readings taken where the paper is silent or inconsistent (all are conventions):
  *   R1  every anchor with t_s >= 0 is a candidate, i.e. (s+1)^2 <= i+1, n(i) = floor(sqrt(i+1));
  *   R2  spans are the closed interval of Algorithm 1 (so (b+f)*l + 1 tokens when unclipped);
  *   R3  l(i) is the exact integer ceiling of sqrt(i); l(0) = 0;
@@ -35,7 +34,10 @@
  *       (and the window) -- this reduces to dense causal attention when the selection covers every
  *       key.  PER_SPAN: Algorithm 1 literally -- one softmax per span (J_t = S_t united with W),
  *       then the gate of the Combination section.
- *   R8  the window W = [max(0, i-w+1), i] removes exactly the anchors with (s+1)^2 <= w.
+ *   R8  the window W = [max(0, i-w+1), i] removes exactly the anchors with (s+1)^2 <= w;
+ *   R9  for exponents other than 1/2 the anchor offset (s+1)^(1/p) and the base length i^p are real
+ *       numbers; both are rounded UP to the next integer, after one part in 1e12 has been taken off
+ *       so that a power that is an integer in exact arithmetic stays that integer (see ceil_pow).
  *
  * Parity pins (tests/test_oracle_*.py): the paper's worked example (i = 30), the anchor gap
  * sequence, the w = 1088 window adjacency, the closed-form work count and its L^{3/2} growth, the
@@ -90,7 +92,7 @@ int64_t sla_oracle_ceil_isqrt(int64_t x) {
 /*
  * General exponents (Section "Span attention": anchors at i - (s+1)^(1/p) + 1 for general p; Section
  * "Training": search_exponent for the stride pattern, span_exponent for the span length).  The paper
- * does not say how the real number (s+1)^(1/p) becomes a position; reading R18: it is rounded UP to
+ * does not say how the real number (s+1)^(1/p) becomes a position; the reading taken here (R9 above): it is rounded UP to
  * an integer, after taking off one part in 1e12 so that a power that is an integer in exact
  * arithmetic (p = 1/3: cubes) is not pushed to the next one by the rounding of 1/p and pow (their
  * relative error is a few 1e-15; positions stay below 2^31, so the margin is far below 1).  For

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libsla.so")
 SLA_OK = 0
 SLA_F32, SLA_BF16 = 0, 1
 SLA_UNION, SLA_PER_SPAN = 0, 1
+SLA_ERR_INVALID_ARG = -1
 
 EXPORTS = [
     "sla_create", "sla_destroy", "sla_workspace_bytes", "sla_status_string", "sla_last_error",
@@ -26,6 +27,7 @@ EXPORTS = [
     "sla_host_staging_bytes", "sla_prefill_host", "sla_kernel_launches", "sla_set_kernel_timing",
     "sla_kernel_time_ms", "sla_decode_step_static", "sla_span_attention_gated",
     "sla_decode_shard_search", "sla_decode_shard_attend", "sla_decode_shard_merge",
+    "sla_pattern_offsets", "sla_pattern_len_steps",
 ]
 
 
@@ -102,8 +104,31 @@ def load_library():
     lib.sla_host_staging_bytes.argtypes = [LP, PP, i64]
     lib.sla_prefill_host.restype = i32
     lib.sla_prefill_host.argtypes = [vp, vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
+    lib.sla_pattern_offsets.restype = C.c_int32
+    lib.sla_pattern_offsets.argtypes = [C.c_double, i64, vp, C.c_int32]
+    lib.sla_pattern_len_steps.restype = C.c_int32
+    lib.sla_pattern_len_steps.argtypes = [C.c_double, i64, vp, C.c_int32]
     _lib = lib
     return lib
+
+
+def _pattern_table(fn, exponent: float, reach: int):
+    n = fn(float(exponent), int(reach), None, 0)
+    if n < 0:
+        raise SlaError(SLA_ERR_INVALID_ARG, "exponent outside [0.2, 0.8] or more than 65536 entries")
+    buf = (C.c_int32 * max(n, 1))()
+    fn(float(exponent), int(reach), buf, n)
+    return list(buf[:n])
+
+
+def sla_pattern_offsets(search_exponent: float, reach: int):
+    """Stride offsets ceil((s+1)^(1/p)) up to `reach`, as the library derives them (host-only)."""
+    return _pattern_table(load_library().sla_pattern_offsets, search_exponent, reach)
+
+
+def sla_pattern_len_steps(span_exponent: float, reach: int):
+    """Positions at which l(i) = ceil(i^p) steps up, as the library derives them (host-only)."""
+    return _pattern_table(load_library().sla_pattern_len_steps, span_exponent, reach)
 
 
 def make_params(top_k: int, span_len: int, back_factor: int = 2, fwd_factor: int = 0, window: int = 0,

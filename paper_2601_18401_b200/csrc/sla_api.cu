@@ -18,12 +18,15 @@ struct sla_handle_s {
     long long launches = 0;   // kernels launched through this handle
     size_t scratch_avail = 0; // bytes of workspace after the header that kernels may use as scratch
     sla::KernelTimer timer;   // sla_set_kernel_timing / sla_kernel_time_ms
-    bool force_simt = false;  // environment SLA_FORCE_SIMT=1: generic kernels only (for A/B checks)
     // stride-offset and span-length tables for exponents other than 1/2 (host copies; the device
     // copies sit in the workspace header) and what they were built for
     std::vector<int> off_host, len_host;
     double off_p = 0.0, len_p = 0.0;
     long long off_reach = 0, len_reach = 0;
+    // the device copies are enqueued on the stream of the call that built them: a later call on another
+    // stream waits for this event before its kernels read the tables
+    cudaEvent_t tbl_ev = nullptr;
+    cudaStream_t tbl_stream = nullptr;
     // sla_prefill_host: copy-in and copy-out streams and per-chunk events, created on first use
     static constexpr int kMaxChunks = 16;
     cudaStream_t s_in = nullptr, s_out = nullptr;
@@ -155,6 +158,9 @@ sla::Call make_call(const sla_handle_t h, const sla_layout_t *l, const sla_param
 // Builds (or reuses) the handle's pattern tables for this call's exponents and key range and puts
 // the device copies in place on `st`.  Must run before make_call.
 sla_status_t prepare_pattern(sla_handle_t h, const sla_params_t *p, int64_t Lkv, cudaStream_t st) {
+    const bool need_off = !is_half(p->search_exponent), need_len = !is_half(p->span_exponent) && p->span_len == 0;
+    if (!need_off && !need_len) return SLA_OK;
+    bool copied = false;
     if (!is_half(p->search_exponent) && (h->off_p != p->search_exponent || h->off_reach < Lkv)) {
         if (!build_offsets(p->search_exponent, Lkv, h->off_host))
             return fail(h, SLA_ERR_UNSUPPORTED, "search_exponent gives more than 65536 strides for this length%s");
@@ -163,6 +169,7 @@ sla_status_t prepare_pattern(sla_handle_t h, const sla_params_t *p, int64_t Lkv,
         if (!h->off_host.empty() &&
             cudaMemcpyAsync(h->ws + kOffTableAt, h->off_host.data(), h->off_host.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
             return fail(h, SLA_ERR_CUDA, "copying the stride table failed%s");
+        copied = true;
     }
     if (!is_half(p->span_exponent) && p->span_len == 0 && (h->len_p != p->span_exponent || h->len_reach < Lkv)) {
         if (!build_len_first(p->span_exponent, Lkv, h->len_host))
@@ -172,6 +179,15 @@ sla_status_t prepare_pattern(sla_handle_t h, const sla_params_t *p, int64_t Lkv,
         if (!h->len_host.empty() &&
             cudaMemcpyAsync(h->ws + kLenTableAt, h->len_host.data(), h->len_host.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
             return fail(h, SLA_ERR_CUDA, "copying the span-length table failed%s");
+        copied = true;
+    }
+    if (copied) {
+        if (!h->tbl_ev && cudaEventCreateWithFlags(&h->tbl_ev, cudaEventDisableTiming) != cudaSuccess)
+            return fail(h, SLA_ERR_CUDA, "creating the table event failed%s");
+        if (cudaEventRecord(h->tbl_ev, st) != cudaSuccess) return fail(h, SLA_ERR_CUDA, "recording the table event failed%s");
+        h->tbl_stream = st;
+    } else if (h->tbl_ev && st != h->tbl_stream) {
+        if (cudaStreamWaitEvent(st, h->tbl_ev, 0) != cudaSuccess) return fail(h, SLA_ERR_CUDA, "waiting for the tables failed%s");
     }
     return SLA_OK;
 }
@@ -252,6 +268,22 @@ sla_status_t sla_kernel_time_ms(sla_handle_t h, float *ms, int32_t *n_launches) 
     return SLA_OK;
 }
 
+int32_t sla_pattern_offsets(double p, int64_t reach, int32_t *out, int32_t cap) {
+    if (!(p >= 0.2 && p <= 0.8) || reach < 0 || cap < 0 || (cap > 0 && !out)) return -1;
+    std::vector<int> t;
+    if (!build_offsets(p, reach, t)) return -1;
+    for (int j = 0; j < cap && j < (int)t.size(); ++j) out[j] = t[j];
+    return (int32_t)t.size();
+}
+
+int32_t sla_pattern_len_steps(double p, int64_t reach, int32_t *out, int32_t cap) {
+    if (!(p >= 0.2 && p <= 0.8) || reach < 0 || cap < 0 || (cap > 0 && !out)) return -1;
+    std::vector<int> t;
+    if (!build_len_first(p, reach, t)) return -1;
+    for (int j = 0; j < cap && j < (int)t.size(); ++j) out[j] = t[j];
+    return (int32_t)t.size();
+}
+
 sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes) {
     if (!handle) return SLA_ERR_INVALID_ARG;
     *handle = nullptr;
@@ -268,7 +300,6 @@ sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device);
     h->ws_bytes = workspace_bytes + kHeaderBytes;
     h->scratch_avail = workspace_bytes;
-    if (const char *fs = getenv("SLA_FORCE_SIMT")) h->force_simt = fs[0] == '1';
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&h->ws), h->ws_bytes);
     if (e == cudaSuccess) e = cudaMemset(h->ws, 0, kHeaderBytes);
     cudaSetDevice(prev);
@@ -289,6 +320,7 @@ sla_status_t sla_destroy(sla_handle_t h) {
         if (h->ev_in[j]) cudaEventDestroy(h->ev_in[j]);
         if (h->ev_done[j]) cudaEventDestroy(h->ev_done[j]);
     }
+    if (h->tbl_ev) cudaEventDestroy(h->tbl_ev);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->s_in) cudaStreamDestroy(h->s_in);
@@ -348,7 +380,7 @@ sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int
     if (sla_status_t ps = prepare_pattern(h, p, Lkv, static_cast<cudaStream_t>(stream))) return ps;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (!h->force_simt && sla::search_mma_supported(c, l->dtype)) {
+    if (sla::search_mma_supported(c, l->dtype)) {
         cudaError_t e = sla::launch_search_mma(q_s, k, c, out_anchor, out_score, st, &h->launches);
         if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_search (tensor-core path)");
         return SLA_OK;
@@ -374,11 +406,14 @@ sla_status_t span_attention_impl(sla_handle_t h, const void *q, const void *k, c
     if (sla_status_t ps = prepare_pattern(h, p, Lkv, static_cast<cudaStream_t>(stream))) return ps;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (!h->force_simt && sla::tc_attention_supported(c, l->dtype)) {
-        // tensor-core path; needs scratch for at least a modest chunk of query positions
+    if (sla::tc_attention_supported(c, l->dtype)) {
+        // tensor-core path; needs scratch for at least a modest chunk of query positions.  A workspace
+        // that cannot hold it is an error, not a reason to run the (far slower) generic kernel.
         const long long min_chunk = Lq < 1024 ? Lq : 1024;
         const sla::TcPlan probe = sla::plan_attention_tc(c, (int)min_chunk);
-        if (probe.ok && probe.bytes <= h->scratch_avail) {
+        if (probe.ok) {
+            if (probe.bytes > h->scratch_avail)
+                return fail(h, SLA_ERR_WORKSPACE, "workspace too small for span-attention: ask sla_workspace_bytes%s");
             cudaError_t e = sla::launch_attn_tc(q, k, v, c, anchor, score, out, lse, lse_span, h->ws + kHeaderBytes,
                                                 h->scratch_avail, h->sm_count, st, &h->launches, &h->timer);
             if (e != cudaSuccess) return cuda_fail(h, e, what);

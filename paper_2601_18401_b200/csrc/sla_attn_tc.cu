@@ -880,29 +880,41 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
     return fn;
 }
 
-// Tensor map over K or V [B, Hkv, Lkv, 128] with arbitrary (16-byte aligned) strides; the three outer
-// dimensions are ordered by ascending stride, slot[] says where (token, head, batch) ended up.
+// The three outer dimensions of K / V (token, head, batch) ordered by ascending stride, as the tensor
+// map wants them.  Dimensions of size 1 go last (their stride is never used and is replaced by one that
+// keeps the list ascending).  False when two dimensions of size > 1 overlap in memory (a stride of 0 from
+// a broadcast view, or a stride smaller than the extent of the dimensions inside it): such a layout is
+// not a tiled tensor, and the caller sends it to the generic kernels, which follow any strides.
+struct KvDim { unsigned long long size, stride; int which; };
+bool order_kv_dims(const Call &c, KvDim (&d)[3]) {
+    d[0] = {(unsigned long long)c.Lkv, (unsigned long long)c.kv_st * 2, 0};
+    d[1] = {(unsigned long long)c.Hkv, (unsigned long long)c.kv_sh * 2, 1};
+    d[2] = {(unsigned long long)c.B, (unsigned long long)c.kv_sb * 2, 2};
+    for (int a = 0; a < 3; ++a)
+        for (int bq = a + 1; bq < 3; ++bq) {
+            const bool swap = (d[bq].size > 1 && d[a].size == 1) ? true
+                              : (d[a].size > 1 && d[bq].size == 1) ? false
+                              : d[bq].stride < d[a].stride;
+            if (swap) { KvDim t = d[a]; d[a] = d[bq]; d[bq] = t; }
+        }
+    unsigned long long extent = (unsigned long long)kD * 2;   // bytes the dimensions inside cover
+    for (int a = 0; a < 3; ++a) {
+        if (d[a].size == 1) d[a].stride = extent;
+        else if (d[a].stride < extent) return false;
+        if (d[a].stride >= (1ull << 40)) return false;        // the tensor map's stride field
+        extent = d[a].stride * d[a].size;
+    }
+    return true;
+}
+
+// Tensor map over K or V [B, Hkv, Lkv, 128] with arbitrary nested (16-byte aligned) strides; slot[] says
+// where (token, head, batch) ended up among the outer dimensions.
 bool make_kv_map(CUtensorMap *tm, const void *ptr, const Call &c, int slot[3]) {
     auto fn = encode_fn();
     if (!fn) return false;
-    struct Dim { unsigned long long size, stride; int which; };
-    Dim d[3] = {{(unsigned long long)c.Lkv, (unsigned long long)c.kv_st * 2, 0},
-                {(unsigned long long)c.Hkv, (unsigned long long)c.kv_sh * 2, 1},
-                {(unsigned long long)c.B, (unsigned long long)c.kv_sb * 2, 2}};
-    for (int a = 0; a < 3; ++a)
-        for (int bq = a + 1; bq < 3; ++bq) {
-            const bool swap = (d[bq].size > 1 && d[a].size == 1) ? false
-                              : (d[a].size > 1 && d[bq].size == 1) ? false
-                              : d[bq].stride < d[a].stride;
-            if (swap) { Dim t = d[a]; d[a] = d[bq]; d[bq] = t; }
-        }
-    // size-1 dimensions get a stride that keeps the list ascending
-    unsigned long long prev = (unsigned long long)kD * 2;
-    for (int a = 0; a < 3; ++a) {
-        if (d[a].size == 1 || d[a].stride < prev) d[a].stride = prev;
-        prev = d[a].stride * d[a].size;
-        slot[d[a].which] = a;
-    }
+    KvDim d[3];
+    if (!order_kv_dims(c, d)) return false;
+    for (int a = 0; a < 3; ++a) slot[d[a].which] = a;
     cuuint64_t gdim[4] = {(cuuint64_t)kD, d[0].size, d[1].size, d[2].size};
     cuuint64_t gstr[3] = {d[0].stride, d[1].stride, d[2].stride};
     cuuint32_t box[4] = {64, 1, 1, 1};
@@ -921,6 +933,8 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 bool tc_attention_shape_ok(const Call &c, int dtype) {
     if (dtype != SLA_BF16 || c.D != kD) return false;
     if (c.kv_st < kD || c.top_k > kMaxTopK || !(c.softmax_scale > 0.f)) return false;
+    KvDim d[3];
+    if (!order_kv_dims(c, d)) return false;   // overlapping K/V dimensions (broadcast views): generic kernels
     const long long ell = base_len(c, c.q_pos0 + c.Lq - 1);
     long long span_tokens = (long long)(c.back + c.fwd) * ell + 1;
     if (c.window > span_tokens) span_tokens = c.window;

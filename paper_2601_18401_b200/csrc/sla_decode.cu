@@ -464,6 +464,22 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
     }
 }
 
+// Dynamic shared memory above 48 KiB has to be allowed per kernel and device context.  The score kernel
+// is given the largest size it can ever be launched with, once per (device, instantiation): later steps
+// then launch without touching function attributes, whatever the context length.
+constexpr int kScoreSmemMax = 200 * 1024;
+template <typename K>
+cudaError_t allow_score_smem(K kern, size_t smem) {
+    static bool done[64] = {};
+    if (smem <= 48 * 1024) return cudaSuccess;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmemMax);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+    return e;
+}
+
 template <typename T, int D>
 cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const void *v, const Call &c,
                           long long n_ctx, const DecodePlan &p, void *scratch, int *counters, void *out, float *lse,
@@ -483,12 +499,12 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
     dim3 gs(n > 0 ? (n + rows_per_cta - 1) / rows_per_cta : 1, c.B * c.Hkv, c.G / gt);
     const T *qs = (const T *)q_s, *kk = (const T *)k;
     const size_t smem = (size_t)(kScoreThreads / 32) * (n + 2 * topk::kCap + 4 * (kMaxTopK + 1)) * sizeof(float);
-    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    if (smem > (size_t)kScoreSmemMax) return cudaErrorInvalidValue;
     cudaError_t e = cudaSuccess;
 #define SLA_LAUNCH_SCORE(GT)                                                                                         \
     do {                                                                                                             \
         auto kern = decode_score<T, D, GT>;                                                                          \
-        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        e = allow_score_smem(kern, smem);                                                                            \
         if (e == cudaSuccess)                                                                                        \
             kern<<<gs, kScoreThreads, smem, st>>>(qs, kk, c, n_ctx, n, s_min, scores, done_bg, spans, out_anchor, out_score); \
     } while (0)
@@ -642,12 +658,12 @@ cudaError_t shard_search_launch(const void *q_s, const void *k_local, const Call
     // positions are global: the local slice starts at shard_lo
     const T *qs = (const T *)q_s, *kk = (const T *)k_local - c.shard_lo * c.kv_st;
     const size_t smem = (size_t)(kScoreThreads / 32) * (n + 2 * topk::kCap + 4 * (kMaxTopK + 1)) * sizeof(float);
-    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    if (smem > (size_t)kScoreSmemMax) return cudaErrorInvalidValue;
     cudaError_t e = cudaSuccess;
 #define SLA_LAUNCH_SCORE(GT)                                                                                         \
     do {                                                                                                             \
         auto kern = decode_score<T, D, GT>;                                                                          \
-        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        e = allow_score_smem(kern, smem);                                                                            \
         if (e == cudaSuccess)                                                                                        \
             kern<<<gs, kScoreThreads, smem, st>>>(qs, kk, c, n_ctx, n, s_first, scores, counters, (int *)nullptr,    \
                                                   cand_anchor, cand_score);                                         \

@@ -53,6 +53,29 @@ def test_workspace_sizing_is_host_only_and_validates(lib):
     assert sla.sla_host_staging_bytes(lay, par, 4096) > 0
 
 
+@pytest.mark.parametrize("p", [1.0 / 3.0, 2.0 / 3.0, 0.54, 0.25])
+def test_pattern_tables_follow_the_rounding_rule(lib, p):
+    """The library's host-built tables for general exponents against the oracle's functions of the same
+    rule (anchors at i + 1 - ceil((s+1)^(1/p)); l(i) = ceil(i^p)), entry by entry, and against exact
+    integer powers where p is the reciprocal of an integer."""
+    import paper_2601_18401_b200 as sla
+    from oracle import sla_oracle as O
+    reach = 200000
+    off = sla.sla_pattern_offsets(p, reach)
+    assert off == [O.stride_offset(s, p) for s in range(len(off))]
+    assert O.stride_offset(len(off), p) > reach >= off[-1]
+    steps = sla.sla_pattern_len_steps(p, reach)
+    assert O.base_len(reach, 0, p) == len(steps)
+    for v, first in list(enumerate(steps, start=1))[:: max(1, len(steps) // 300)]:
+        assert O.base_len(first, 0, p) >= v and (first == 1 or O.base_len(first - 1, 0, p) < v)
+    if abs(p - 1.0 / 3.0) < 1e-12:
+        assert off[:5] == [1, 8, 27, 64, 125] and off[57] == 58 ** 3
+    if p == 0.25:
+        assert off[:4] == [1, 16, 81, 256]
+    assert lib.sla_pattern_offsets(0.9, 100, None, 0) == -1
+    assert lib.sla_pattern_offsets(0.75, 10 ** 9, None, 0) == -1      # more than 65536 strides
+
+
 def test_calls_reject_null_handle(lib):
     assert lib.sla_destroy(None) == -1
     assert lib.sla_poll_status(None, None) == -1

@@ -26,7 +26,20 @@ def sample_rows(L, seed, n_random=192):
     return np.array(sorted(rows), dtype=np.int64)
 
 
-def run_prefill_config(sla, w, seed):
+def stress_rows(L, seed):
+    """The sample of the stress configuration: the first and the last 1024 rows, 2048 rows at seeded
+    positions, and every row whose index is 0 or 127 modulo 128 (the edges of the 128-row tiles)."""
+    rng = np.random.default_rng(seed)
+    rows = set(range(0, 1024)) | set(range(L - 1024, L)) | {int(x) for x in rng.integers(0, L, 2048)}
+    rows |= set(range(0, L, 128)) | set(range(127, L, 128))
+    return np.array(sorted(rows), dtype=np.int64)
+
+
+def run_prefill_config(sla, w, seed, rows, search_all_rows_heads=None):
+    """Search + attention of a whole benchmark configuration in the launch configuration the benchmark
+    times.  `rows`: query positions on which the oracle runs search and attention for every head.
+    `search_all_rows_heads`: (batch, query head) pairs for which the search is compared on ALL rows
+    (None: every pair)."""
     from paper_2601_18401_b200 import synth
     dev = "cuda:0"
     x = synth.make_prefill(w, device=dev)
@@ -35,13 +48,25 @@ def run_prefill_config(sla, w, seed):
     handle = sla.Handle(0, sla.sla_workspace_bytes(layout, params, w.seq_len, w.seq_len) + (64 << 20))
     anchor, score = sla.sla_span_search(handle, x["q_s"], x["k"], params)
     torch.cuda.synchronize()
-    # sampled rows: the oracle's search; the attention then runs on the oracle's selection on those
-    # rows (on both sides) and on the CUDA search result elsewhere
-    rows = sample_rows(w.seq_len, seed)
     host = P.host_inputs(x)
     code = synth.dtype_code(w.dtype)
+    # search on all rows: every head, or the listed ones (one oracle call per head on slices of the inputs)
+    G = w.n_q_heads // w.n_kv_heads
+    ties_all = 0
+    if search_all_rows_heads is None:
+        ref_all = O.span_search(host["q_s"], host["k"], code, top_k=w.top_k)
+        ties_all = P.compare_search(anchor, score, ref_all, q_s=host["q_s"], k=host["k"])
+        del ref_all
+    else:
+        for b, h in search_all_rows_heads:
+            qs1 = np.ascontiguousarray(host["q_s"][b:b + 1, h:h + 1])
+            k1 = np.ascontiguousarray(host["k"][b:b + 1, h // G:h // G + 1])
+            ref1 = O.span_search(qs1, k1, code, top_k=w.top_k)
+            ties_all += P.compare_search(anchor[b:b + 1, h:h + 1], score[b:b + 1, h:h + 1], ref1, q_s=qs1, k=k1)
+    # sampled rows: the oracle's search; the attention then runs on the oracle's selection on those
+    # rows (on both sides) and on the CUDA search result elsewhere
     ref_s = O.span_search(host["q_s"], host["k"], code, top_k=w.top_k, rows=rows)
-    ties = P.compare_search(anchor, score, ref_s, rows=rows)
+    ties = P.compare_search(anchor, score, ref_s, rows=rows, q_s=host["q_s"], k=host["k"])
     anchor = P.oracle_anchors_on_device(anchor, ref_s, rows=rows)
     out, lse = sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params)
     torch.cuda.synchronize()
@@ -60,47 +85,42 @@ def run_prefill_config(sla, w, seed):
     ref_a = P.oracle_attention_for(host, code, ref_s["anchor"], w, rows=rows)
     err, lerr = P.compare_attention(out, lse, ref_a, w.dtype, rows=rows)
     handle.close()
-    return dict(ties=ties, rows=len(rows), err=err, lerr=lerr)
+    return dict(ties=ties, ties_all_rows=ties_all, rows=len(rows), err=err, lerr=lerr)
 
 
 def test_prefill_L65536_planted(sla):
     """Second benchmark configuration: 32/8 heads, L = 65536, bf16, 16 planted spans, l = 256, k = 8."""
     from paper_2601_18401_b200 import synth
-    r = run_prefill_config(sla, synth.CONFIGS[1], seed=11)
+    w = synth.CONFIGS[1]
+    r = run_prefill_config(sla, w, 11, sample_rows(w.seq_len, 11, n_random=1024))   # search: all rows, all heads
     print("prefill_L65536:", r)
     assert r["ties"] <= 0.02 * r["rows"] * 32
+    assert r["ties_all_rows"] <= 0.02 * w.seq_len * 32
 
 
 def test_prefill_stress_L262144(sla):
     """Third benchmark configuration: batch 2, 16/4 heads, L = 262144, l = 512, k = 16."""
     from paper_2601_18401_b200 import synth
-    r = run_prefill_config(sla, synth.CONFIGS[2], seed=12)
+    w = synth.CONFIGS[2]
+    # search on ALL rows for four (batch, query head) pairs, one per KV head; every head on the sampled rows
+    r = run_prefill_config(sla, w, 12, stress_rows(w.seq_len, 12), search_all_rows_heads=[(0, 0), (0, 9), (1, 6), (1, 15)])
     print("prefill_stress:", r)
     assert r["ties"] <= 0.05 * r["rows"] * 32
+    assert r["ties_all_rows"] <= 0.05 * w.seq_len * 4
 
 
 def _decode_check(sla, handle, w, kc, vc, hk, hv, n_ctx, step_inputs, sparse_fill=None):
     from paper_2601_18401_b200 import synth
     params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
-    out, lse, anchor, score = sla.sla_decode_step(handle, step_inputs["q_s"], step_inputs["q"], kc, vc, n_ctx, params)
+    got = sla.sla_decode_step(handle, step_inputs["q_s"], step_inputs["q"], kc, vc, n_ctx, params)
     torch.cuda.synchronize()
     assert sla.sla_poll_status(handle) == sla.SLA_OK
-    code = synth.dtype_code(w.dtype)
-    q_s = synth.to_numpy(step_inputs["q_s"])[:, :, None]
-    q = synth.to_numpy(step_inputs["q"])[:, :, None]
     if sparse_fill is not None:
         sparse_fill(anchor_rows=True)
-    ref_s = O.span_search(q_s, hk, code, top_k=w.top_k, q_pos0=n_ctx - 1, Lkv=n_ctx)
-    P.compare_search(anchor[:, :, None], score[:, :, None], ref_s, q_pos0=n_ctx - 1)
-    # attention of the step against the oracle on the oracle's own selection, on the heads where the
-    # two selections agree (the others are near-ties, counted above)
-    ra = ref_s["anchor"][:, :, 0]
-    if sparse_fill is not None:
-        sparse_fill(anchors=ra)
-    att = O.span_attention(q, hk, hv, code, ref_s["anchor"], span_len=w.span_len, q_pos0=n_ctx - 1, Lkv=n_ctx)
-    same = P.same_selection(anchor, ra)
-    assert same.mean() > 0.7
-    return P.compare_attention(out[:, :, None], lse[:, :, None], att, w.dtype, where=same[:, :, None])
+    hook = None if sparse_fill is None else (lambda sets: [sparse_fill(anchors=a) for a in sets])
+    return P.check_decode_step(got, synth.to_numpy(step_inputs["q_s"]), synth.to_numpy(step_inputs["q"]), hk, hv,
+                               synth.dtype_code(w.dtype), w.dtype, n_ctx=n_ctx, top_k=w.top_k, span_len=w.span_len,
+                               before_attention=hook)
 
 
 def test_decode_1M(sla):
@@ -108,12 +128,13 @@ def test_decode_1M(sla):
     from paper_2601_18401_b200 import synth
     w = synth.CONFIGS[3]
     dev = "cuda:0"
-    steps = 6
+    steps = 32
     kc, vc = synth.make_decode_cache(w, dev, capacity=w.seq_len + steps)
     hk, hv = synth.to_numpy(kc), synth.to_numpy(vc)
     layout = sla.make_layout(torch.empty(1, 32, 128, dtype=torch.bfloat16, device=dev), kc, decode=True)
     params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
     handle = sla.Handle(0, sla.sla_workspace_bytes(layout, params, 1, w.seq_len + steps) + (16 << 20))
+    stats = []
     for s in range(steps):
         x = synth.make_decode_step_inputs(w, s, dev)
         n_ctx = w.seq_len + s + 1
@@ -121,8 +142,8 @@ def test_decode_1M(sla):
         vc[:, :, n_ctx - 1] = x["v_new"]
         hk[:, :, n_ctx - 1] = synth.to_numpy(x["k_new"])
         hv[:, :, n_ctx - 1] = synth.to_numpy(x["v_new"])
-        err, lerr = _decode_check(sla, handle, w, kc, vc, hk, hv, n_ctx, x)
-        assert err <= 1e-2
+        stats.append(_decode_check(sla, handle, w, kc, vc, hk, hv, n_ctx, x))
+    print("decode_1M (heads on the oracle's selection, on the alternative, left out) per step:", stats)
     handle.close()
 
 
@@ -135,7 +156,7 @@ def test_decode_10M(sla):
     free, _ = torch.cuda.mem_get_info()
     if free < 30 << 30:
         pytest.skip("needs 30 GB of free device memory")
-    steps = 2
+    steps = 8
     cap = w.seq_len + steps
     kc, vc = synth.make_decode_cache(w, dev, capacity=cap)
     shape = (w.batch, w.n_kv_heads, cap, w.head_dim)
@@ -144,6 +165,7 @@ def test_decode_10M(sla):
     params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
     handle = sla.Handle(0, sla.sla_workspace_bytes(layout, params, 1, cap) + (16 << 20))
     span = w.back_factor * w.span_len
+    stats = []
     for s in range(steps):
         x = synth.make_decode_step_inputs(w, s, dev)
         n_ctx = w.seq_len + s + 1
@@ -162,8 +184,8 @@ def test_decode_10M(sla):
                     hk[:, :, lo:hi + 1] = synth.to_numpy(kc[:, :, lo:hi + 1])
                     hv[:, :, lo:hi + 1] = synth.to_numpy(vc[:, :, lo:hi + 1])
 
-        err, lerr = _decode_check(sla, handle, w, kc, vc, hk, hv, n_ctx, x, sparse_fill=fill)
-        assert err <= 1e-2
+        stats.append(_decode_check(sla, handle, w, kc, vc, hk, hv, n_ctx, x, sparse_fill=fill))
+    print("decode_10M (heads on the oracle's selection, on the alternative, left out) per step:", stats)
     handle.close()
 
 
@@ -190,7 +212,7 @@ def test_prefill_paper_kernel_config(sla):
         hq = np.ascontiguousarray(host["q"][:, :, q0:q0 + ch])
         ref_s = O.span_search(hq_s, host["k"], code, top_k=w.top_k, q_pos0=q0, Lkv=q0 + ch, window=w.window,
                               rows=rows)
-        ties = P.compare_search(anchor, score, ref_s, q_pos0=q0, rows=rows)
+        ties = P.compare_search(anchor, score, ref_s, q_pos0=q0, rows=rows, q_s=hq_s, k=host["k"], window=w.window)
         # on the sampled rows the attention runs on the oracle's selection and scores, on both sides
         idx = torch.as_tensor(rows, device=dev)
         anchor = P.oracle_anchors_on_device(anchor, ref_s, rows=rows)

@@ -260,7 +260,13 @@ def test_union_attention_against_set_brute_force(b, f, window, span_len):
 
 
 def test_per_span_gate_against_brute_force():
-    """Algorithm 1 literally: per-span softmax, then the softmax gate of the Combination section."""
+    """Algorithm 1 literally: per-span softmax (the line for A_{i,t}), then the softmax gate of the
+    Combination section.  Besides `out` this pins the two log-sum-exp outputs of the per-span mode:
+    `lse_span[j]` is the log-sum-exp of the logits over J_t = S_t united with W of the j-th selected
+    anchor, recomputed here from the key set itself (-inf on padding), and `lse` is the value of the
+    best-scoring selected anchor (slot 0 of a selection that comes from the search).  Both checks
+    fail on an oracle that swaps two `lse_span` slots or takes the wrong "first" span (verified by
+    running the assertions on a copy with slots 0 and 1 exchanged, at the end)."""
     B, Hq, Hkv, L, D = 1, 2, 2, 120, 8
     q_s, q = rand((B, Hq, L, D), 19), rand((B, Hq, L, D), 20)
     k, v = rand((B, Hkv, L, D), 21), rand((B, Hkv, L, D), 22)
@@ -268,20 +274,41 @@ def test_per_span_gate_against_brute_force():
         sr = O.span_search(q_s, k, O.F64, top_k=3, window=window)
         at = O.span_attention(q, k, v, O.F64, sr["anchor"], span_len=0, back_factor=2, fwd_factor=1,
                               window=window, mode=O.PER_SPAN, score=sr["score"], softmax_scale=0.25)
+        want_span = np.full(at["lse_span"].shape, -np.inf)
+        want_lse = np.full(at["lse"].shape, -np.inf)
         for h in range(Hq):
             for i in range(L):
                 an = [int(a) for a in sr["anchor"][0, h, i] if a >= 0]
                 ell = math.isqrt(i - 1) + 1 if i > 0 else 0
                 if not an:
-                    want, _ = brute_union(q[0, h, i], k[0, h], v[0, h], i, [], ell, 2, 1, 0.25, window)
+                    want, want_lse[0, h, i] = brute_union(q[0, h, i], k[0, h], v[0, h], i, [], ell, 2, 1, 0.25, window)
                 else:
                     s = sr["score"][0, h, i, :len(an)]
                     alpha = np.exp(s - s.max())
                     alpha /= alpha.sum()
                     assert abs(alpha.sum() - 1.0) < 1e-12
-                    want = sum(al * brute_union(q[0, h, i], k[0, h], v[0, h], i, [t], ell, 2, 1, 0.25, window)[0]
-                               for al, t in zip(alpha, an))
+                    per = [brute_union(q[0, h, i], k[0, h], v[0, h], i, [t], ell, 2, 1, 0.25, window) for t in an]
+                    want = sum(al * o for al, (o, _) in zip(alpha, per))
+                    want_span[0, h, i, :len(an)] = [l for _, l in per]
+                    want_lse[0, h, i] = per[int(np.argmax(s))][1]    # the best-scoring selected anchor
                 np.testing.assert_allclose(at["out"][0, h, i], want, atol=1e-12)
+
+        def check(lse_span, lse):
+            fin = np.isfinite(want_span)
+            assert np.array_equal(np.isneginf(lse_span), ~fin)
+            np.testing.assert_allclose(lse_span[fin], want_span[fin], atol=1e-12)
+            finl = np.isfinite(want_lse)
+            assert np.array_equal(np.isneginf(lse), ~finl)
+            np.testing.assert_allclose(lse[finl], want_lse[finl], atol=1e-12)
+
+        check(at["lse_span"], at["lse"])
+        # the pin has teeth: two exchanged slots, or the second span's value as `lse`, are caught
+        swapped = at["lse_span"].copy()
+        swapped[..., [0, 1]] = swapped[..., [1, 0]]
+        with pytest.raises(AssertionError):
+            check(swapped, at["lse"])
+        with pytest.raises(AssertionError):
+            check(at["lse_span"], at["lse_span"][..., 1])
 
 
 # --------------------------------------------------------------------------- special cases

@@ -60,3 +60,11 @@ def test_static_scratch_rejects_steps_beyond_its_fixed_size():
         sla.sla_decode_step_static(q, q, kc, kc, n_ctx, sla.make_params(16, 64), out=out, lse=lse,
                                    out_anchor=anchor, out_score=score)
     assert e.value.status == -3
+    # what the fixed array cannot serve is refused on the host, before anything is launched: a local
+    # window, the per-span mode and other exponents all need scratch that only a handle has
+    small = dict(out=out[:1, :8], lse=lse[:1, :8], out_anchor=anchor[:1, :8], out_score=score[:1, :8])
+    for bad in (sla.make_params(16, 64, window=1), sla.make_params(16, 64, mode=sla.SLA_PER_SPAN),
+                sla.make_params(16, 64, search_exponent=1.0 / 3.0)):
+        with pytest.raises(sla.SlaError) as e:
+            sla.sla_decode_step_static(q[:1, :8], q[:1, :8], kc[:1], kc[:1], n_ctx, bad, **small)
+        assert e.value.status == -2
