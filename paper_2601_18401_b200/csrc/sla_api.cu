@@ -380,6 +380,11 @@ sla_status_t sla_span_search(sla_handle_t h, const void *q_s, const void *k, int
     if (sla_status_t ps = prepare_pattern(h, p, Lkv, static_cast<cudaStream_t>(stream))) return ps;
     sla::Call c = make_call(h, l, p, Lq, q_pos0, Lkv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (sla::search_diag_supported(c, l->dtype) && ((reinterpret_cast<uintptr_t>(q_s) | reinterpret_cast<uintptr_t>(k)) & 31u) == 0) {
+        cudaError_t e = sla::launch_search_diag(q_s, k, c, out_anchor, out_score, st, &h->launches);
+        if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_search (fused selection)");
+        return SLA_OK;
+    }
     if (sla::search_mma_supported(c, l->dtype)) {
         cudaError_t e = sla::launch_search_mma(q_s, k, c, out_anchor, out_score, st, &h->launches);
         if (e != cudaSuccess) return cuda_fail(h, e, "sla_span_search (tensor-core path)");

@@ -27,6 +27,12 @@ bool search_mma_supported(const Call &c, int dtype);
 cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int32_t *out_anchor, float *out_score,
                               cudaStream_t st, long long *launches);
 
+// ---- span-search with the selection folded into the scoring loop, bf16 / head_dim 128 / groups of four
+// query heads (sla_search_diag.cu)
+bool search_diag_supported(const Call &c, int dtype);
+cudaError_t launch_search_diag(const void *q_s, const void *k, const Call &c, int32_t *out_anchor, float *out_score,
+                               cudaStream_t st, long long *launches);
+
 // ---- tensor-core span-attention for prefill, bf16 / head_dim 128 (sla_attn_tc.cu) ---------------
 // Scratch layout for one chunk of Lc query positions (all offsets in bytes).
 struct TcPlan {

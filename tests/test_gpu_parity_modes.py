@@ -81,6 +81,7 @@ def run_modes(sla, handle, w, window, q_pos0=0):
     dict(top_k=40, seq_len=300, span_len=5),                       # padding; rows with nothing selected
     dict(top_k=8, span_len=10, seq_len=777),                       # the largest k of the row-parallel gated merge
     dict(top_k=9, span_len=10, seq_len=777),                       # the smallest k of the general one
+    dict(n_q_heads=8, n_kv_heads=2, top_k=6, span_len=14, seq_len=1400),   # groups of four query heads
 ])
 def test_modes_and_window(sla, handle, kw, window):
     run_modes(sla, handle, workload(**kw), window)
@@ -168,6 +169,7 @@ def run_exponents(sla, handle, w, p_search, p_span, window=0, mode="union", top_
     dict(span_len=0, top_k=3),                                          # bf16 D128 GQA, l(i) from the exponent
     dict(span_len=0, dtype="f32", head_dim=64, n_q_heads=2, n_kv_heads=1, seq_len=600, top_k=2),
     dict(span_len=12, top_k=4),                                         # fixed base length
+    dict(span_len=0, top_k=5, n_q_heads=8, n_kv_heads=2, seq_len=1300),  # groups of four query heads
 ])
 def test_general_exponents(sla, handle, kw, p_search, p_span):
     run_exponents(sla, handle, workload(**kw), p_search, p_span)

