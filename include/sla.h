@@ -70,7 +70,8 @@ typedef enum {
     SLA_ERR_WORKSPACE = -3,      /* the handle's workspace is too small for this call             */
     SLA_ERR_CUDA = -4,           /* a CUDA runtime call failed (see sla_last_error)               */
     SLA_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait expired                            */
-    SLA_ERR_DEVICE_INDEX = -6    /* a kernel met an anchor outside [0, i] and skipped it          */
+    SLA_ERR_DEVICE_INDEX = -6,   /* a kernel met an anchor outside [0, i] and skipped it          */
+    SLA_ERR_DEVICE_OVERRUN = -7  /* debug canaries: a kernel wrote outside its scratch region      */
 } sla_status_t;
 
 typedef enum { SLA_F32 = 0, SLA_BF16 = 1 } sla_dtype_t;
@@ -132,8 +133,8 @@ size_t sla_workspace_bytes(const sla_layout_t *layout, const sla_params_t *param
 const char *sla_status_string(sla_status_t status); /* static string, never NULL                  */
 const char *sla_last_error(sla_handle_t handle);    /* text of the last failure on this handle     */
 
-/* Waits for `stream` and reads the device status word: SLA_OK, SLA_ERR_DEVICE_TIMEOUT or
- * SLA_ERR_DEVICE_INDEX; the word is cleared. */
+/* Waits for `stream` and reads the device status word: SLA_OK, SLA_ERR_DEVICE_OVERRUN,
+ * SLA_ERR_DEVICE_TIMEOUT or SLA_ERR_DEVICE_INDEX; the word is cleared. */
 sla_status_t sla_poll_status(sla_handle_t handle, void *stream);
 
 /* Number of kernels this handle has launched since sla_create (a diagnostic for benchmarks; the
@@ -147,6 +148,34 @@ int64_t sla_kernel_launches(sla_handle_t handle);
  * the previous read and how many they were (n_launches may be NULL), and starts over. */
 sla_status_t sla_set_kernel_timing(sla_handle_t handle, int enable);
 sla_status_t sla_kernel_time_ms(sla_handle_t handle, float *ms, int32_t *n_launches);
+
+/* Debug canaries (the paper has no counterpart; they stand in for a memory checker).  When enabled,
+ * sla_span_attention, sla_span_attention_gated and sla_decode_step separate the regions of their scratch
+ * memory by 256-byte gaps, fill the gaps with a pattern before their kernels run and check them
+ * afterwards; a damaged gap shows as SLA_ERR_DEVICE_OVERRUN at the next sla_poll_status.  Costs two
+ * small launches per call (per chunk of a chunked call); off by default.
+ * sla_selftest_canary_trip damages one gap of the most recent sla_decode_step of this handle itself (a
+ * 4-byte memset, nothing out of bounds) and runs the check again, to show that the check reports. */
+sla_status_t sla_set_debug_canaries(sla_handle_t handle, int enable);
+sla_status_t sla_selftest_canary_trip(sla_handle_t handle, void *stream);
+
+/* Read-only L2 bandwidth probe (a diagnostic for benchmarks; the paper has no counterpart): every CTA of
+ * a grid of 4 x SM count reads the whole device buffer `buf` (`bytes`: a multiple of 8192, small enough
+ * to stay resident in L2) `iters` times with 32-byte loads, the access width of the span-search kernel,
+ * whose roofline this bandwidth is (key rows stream out of L2).  Bytes read by one call:
+ * 4 * SM count * bytes * iters.  The caller times the call with CUDA events on `stream`.  `sink`: four
+ * bytes of device memory or NULL (never written in practice; it keeps the loads alive). */
+sla_status_t sla_probe_l2_read(sla_handle_t handle, const void *buf, size_t bytes, int32_t iters, void *sink,
+                               void *stream);
+
+/* Self-test of the bounded device-side wait (the paper has no counterpart).  Launches one warp that polls
+ * a barrier nothing ever arrives on, at most `max_polls` (1 .. 10000) times -- no copy and no MMA is in
+ * flight -- then records the time-out in the status word, exactly as the tensor-core kernels do when
+ * one of their waits runs out, and returns by itself.  The next sla_poll_status reports
+ * SLA_ERR_DEVICE_TIMEOUT once; the handle stays usable.  polls_done_device: optional device int that
+ * receives the number of polls made. */
+sla_status_t sla_selftest_wait_expiry(sla_handle_t handle, int32_t max_polls, int32_t *polls_done_device,
+                                      void *stream);
 
 /* The two integer tables the library derives from exponents other than 1/2 (host-only diagnostics, so
  * that the rounding rule stated at sla_params_t can be checked without a device; Section "Span

@@ -27,7 +27,8 @@ EXPORTS = [
     "sla_host_staging_bytes", "sla_prefill_host", "sla_kernel_launches", "sla_set_kernel_timing",
     "sla_kernel_time_ms", "sla_decode_step_static", "sla_span_attention_gated",
     "sla_decode_shard_search", "sla_decode_shard_attend", "sla_decode_shard_merge",
-    "sla_pattern_offsets", "sla_pattern_len_steps",
+    "sla_pattern_offsets", "sla_pattern_len_steps", "sla_probe_l2_read", "sla_selftest_wait_expiry",
+    "sla_set_debug_canaries", "sla_selftest_canary_trip",
 ]
 
 
@@ -104,6 +105,14 @@ def load_library():
     lib.sla_host_staging_bytes.argtypes = [LP, PP, i64]
     lib.sla_prefill_host.restype = i32
     lib.sla_prefill_host.argtypes = [vp, vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
+    lib.sla_set_debug_canaries.restype = i32
+    lib.sla_set_debug_canaries.argtypes = [vp, i32]
+    lib.sla_selftest_canary_trip.restype = i32
+    lib.sla_selftest_canary_trip.argtypes = [vp, vp]
+    lib.sla_probe_l2_read.restype = i32
+    lib.sla_probe_l2_read.argtypes = [vp, vp, sz, C.c_int32, vp, vp]
+    lib.sla_selftest_wait_expiry.restype = i32
+    lib.sla_selftest_wait_expiry.argtypes = [vp, C.c_int32, vp, vp]
     lib.sla_pattern_offsets.restype = C.c_int32
     lib.sla_pattern_offsets.argtypes = [C.c_double, i64, vp, C.c_int32]
     lib.sla_pattern_len_steps.restype = C.c_int32
@@ -221,6 +230,31 @@ def sla_kernel_time_ms(handle: Handle):
     ms, n = C.c_float(0.0), C.c_int32(0)
     handle.check(handle._lib.sla_kernel_time_ms(handle.ptr, C.byref(ms), C.byref(n)), "sla_kernel_time_ms")
     return float(ms.value), int(n.value)
+
+
+def sla_set_debug_canaries(handle: Handle, enable: bool) -> None:
+    handle.check(handle._lib.sla_set_debug_canaries(handle.ptr, int(bool(enable))), "sla_set_debug_canaries")
+
+
+def sla_selftest_canary_trip(handle: Handle, stream=None) -> None:
+    handle.check(handle._lib.sla_selftest_canary_trip(handle.ptr, _stream_ptr(stream)), "sla_selftest_canary_trip")
+
+
+def sla_probe_l2_read(handle: Handle, buf: torch.Tensor, iters: int, stream=None) -> int:
+    """Launches the read-only L2 probe over `buf` (device, contiguous); returns the bytes it reads."""
+    nbytes = buf.numel() * buf.element_size()
+    handle.check(handle._lib.sla_probe_l2_read(handle.ptr, buf.data_ptr(), nbytes, int(iters), None, _stream_ptr(stream)),
+                 "sla_probe_l2_read")
+    sms = torch.cuda.get_device_properties(buf.device).multi_processor_count
+    return 4 * sms * nbytes * int(iters)
+
+
+def sla_selftest_wait_expiry(handle: Handle, max_polls: int = 2000, polls_done: Optional[torch.Tensor] = None,
+                             stream=None) -> None:
+    """Makes a bounded device-side wait run out on purpose-built barrier nothing arrives on (see sla.h)."""
+    handle.check(handle._lib.sla_selftest_wait_expiry(handle.ptr, int(max_polls),
+                                                     None if polls_done is None else polls_done.data_ptr(),
+                                                     _stream_ptr(stream)), "sla_selftest_wait_expiry")
 
 
 def sla_poll_status(handle: Handle, stream=None) -> int:

@@ -18,6 +18,9 @@ struct sla_handle_s {
     long long launches = 0;   // kernels launched through this handle
     size_t scratch_avail = 0; // bytes of workspace after the header that kernels may use as scratch
     sla::KernelTimer timer;   // sla_set_kernel_timing / sla_kernel_time_ms
+    bool canaries = false;    // sla_set_debug_canaries
+    sla::Canaries last_canaries;   // of the most recent call that laid any, and where its scratch began
+    char *last_canary_base = nullptr;
     // stride-offset and span-length tables for exponents other than 1/2 (host copies; the device
     // copies sit in the workspace header) and what they were built for
     std::vector<int> off_host, len_host;
@@ -234,6 +237,7 @@ const char *sla_status_string(sla_status_t s) {
         case SLA_ERR_CUDA: return "SLA_ERR_CUDA";
         case SLA_ERR_DEVICE_TIMEOUT: return "SLA_ERR_DEVICE_TIMEOUT";
         case SLA_ERR_DEVICE_INDEX: return "SLA_ERR_DEVICE_INDEX";
+        case SLA_ERR_DEVICE_OVERRUN: return "SLA_ERR_DEVICE_OVERRUN";
     }
     return "SLA_ERR_UNKNOWN";
 }
@@ -282,6 +286,52 @@ int32_t sla_pattern_len_steps(double p, int64_t reach, int32_t *out, int32_t cap
     if (!build_len_first(p, reach, t)) return -1;
     for (int j = 0; j < cap && j < (int)t.size(); ++j) out[j] = t[j];
     return (int32_t)t.size();
+}
+
+sla_status_t sla_set_debug_canaries(sla_handle_t h, int enable) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    h->canaries = enable != 0;
+    h->last_canaries = sla::Canaries();
+    h->last_canary_base = nullptr;
+    return SLA_OK;
+}
+
+sla_status_t sla_selftest_canary_trip(sla_handle_t h, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (!h->last_canary_base || h->last_canaries.n == 0)
+        return fail(h, SLA_ERR_INVALID_ARG, "no decode step with canaries has run on this handle%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // what an overrun of the first scratch region by one word would leave behind
+    cudaError_t e = cudaMemsetAsync(h->last_canary_base + h->last_canaries.at[1], 0, 4, st);
+    if (e == cudaSuccess) e = sla::launch_canary_check(h->last_canary_base, h->last_canaries, reinterpret_cast<int *>(h->ws), st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_selftest_canary_trip");
+    return SLA_OK;
+}
+
+sla_status_t sla_probe_l2_read(sla_handle_t h, const void *buf, size_t bytes, int32_t iters, void *sink, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (!buf || !aligned16(buf) || (reinterpret_cast<uintptr_t>(buf) & 31u) || iters < 1 || iters > 4096)
+        return fail(h, SLA_ERR_INVALID_ARG, "probe buffer must be 32-byte aligned, iters in 1..4096%s");
+    if (bytes < 8192 || bytes % 8192 || bytes > ((size_t)1 << 32))
+        return fail(h, SLA_ERR_INVALID_ARG, "probe size must be a multiple of 8192 bytes, at most 4 GiB%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    cudaError_t e = sla::launch_probe_l2_read(buf, bytes, iters, 4 * h->sm_count, static_cast<unsigned *>(sink),
+                                              static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_probe_l2_read");
+    h->launches += 1;
+    return SLA_OK;
+}
+
+sla_status_t sla_selftest_wait_expiry(sla_handle_t h, int32_t max_polls, int32_t *polls_done_device, void *stream) {
+    if (!h) return SLA_ERR_INVALID_ARG;
+    if (max_polls < 1 || max_polls > 10000) return fail(h, SLA_ERR_INVALID_ARG, "max_polls must be in 1..10000%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    cudaError_t e = sla::launch_selftest_wait_expiry(max_polls, reinterpret_cast<int *>(h->ws), polls_done_device,
+                                                     static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_selftest_wait_expiry");
+    h->launches += 1;
+    return SLA_OK;
 }
 
 sla_status_t sla_create(sla_handle_t *handle, int device, size_t workspace_bytes) {
@@ -352,7 +402,7 @@ size_t sla_workspace_bytes(const sla_layout_t *l, const sla_params_t *p, int64_t
         const sla::TcPlan tp = sla::plan_attention_tc(c, (int)(Lq < 65536 ? Lq : 65536));
         if (tp.bytes > need) need = tp.bytes;
     }
-    return need + 4096;
+    return need + 4096 + (sla::Canaries::kMax + 1) * sla::Canaries::kBytes;   // slack, and room for debug canaries
 }
 
 sla_status_t sla_poll_status(sla_handle_t h, void *stream) {
@@ -363,6 +413,7 @@ sla_status_t sla_poll_status(sla_handle_t h, void *stream) {
     if (e == cudaSuccess) e = cudaMemsetAsync(h->ws, 0, sizeof word, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_poll_status");
+    if (word & sla::kStatusOverrun) return fail(h, SLA_ERR_DEVICE_OVERRUN, "a kernel wrote outside its scratch region%s");
     if (word & sla::kStatusTimeout) return fail(h, SLA_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired%s");
     if (word & sla::kStatusBadIndex) return fail(h, SLA_ERR_DEVICE_INDEX, "an anchor outside [0, i] was skipped%s");
     return SLA_OK;
@@ -415,12 +466,12 @@ sla_status_t span_attention_impl(sla_handle_t h, const void *q, const void *k, c
         // tensor-core path; needs scratch for at least a modest chunk of query positions.  A workspace
         // that cannot hold it is an error, not a reason to run the (far slower) generic kernel.
         const long long min_chunk = Lq < 1024 ? Lq : 1024;
-        const sla::TcPlan probe = sla::plan_attention_tc(c, (int)min_chunk);
+        const sla::TcPlan probe = sla::plan_attention_tc(c, (int)min_chunk, h->canaries ? sla::Canaries::kBytes : 0);
         if (probe.ok) {
             if (probe.bytes > h->scratch_avail)
                 return fail(h, SLA_ERR_WORKSPACE, "workspace too small for span-attention: ask sla_workspace_bytes%s");
             cudaError_t e = sla::launch_attn_tc(q, k, v, c, anchor, score, out, lse, lse_span, h->ws + kHeaderBytes,
-                                                h->scratch_avail, h->sm_count, st, &h->launches, &h->timer);
+                                                h->scratch_avail, h->sm_count, st, &h->launches, &h->timer, h->canaries);
             if (e != cudaSuccess) return cuda_fail(h, e, what);
             return SLA_OK;
         }
@@ -471,17 +522,22 @@ sla_status_t sla_decode_step(sla_handle_t h, const void *q_s, const void *q, con
     if (sla_status_t ps = prepare_pattern(h, p, n_ctx, static_cast<cudaStream_t>(stream))) return ps;
     sla::Call c = make_call(h, l, p, 1, n_ctx - 1, n_ctx);
     const sla::DecodePlan plan =
-        sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim));
+        sla::plan_decode(c, n_ctx, h->sm_count * sla::decode_attn_blocks_per_sm(l->dtype, l->head_dim),
+                         h->canaries ? sla::Canaries::kBytes : 0);
     if (plan.bytes + kHeaderBytes > h->ws_bytes) return fail(h, SLA_ERR_WORKSPACE, "workspace too small for this decode step%s");
     if ((size_t)plan.n_anchor * sizeof(float) * 8 > 180 * 1024) return fail(h, SLA_ERR_UNSUPPORTED, "context too long for the decode top-k stage%s");
     const size_t units = p->mode == SLA_PER_SPAN ? (size_t)p->top_k : 1;
     if ((size_t)(l->batch) * (l->n_kv_heads + l->n_q_heads * (units + 1)) * sizeof(int) > kCounterEnd - kCounterOffset)
         return fail(h, SLA_ERR_UNSUPPORTED, "too many (batch, head) pairs for the decode step%s");
-    cudaError_t e = sla::launch_decode(q_s, q, k_cache, v_cache, c, l->dtype, n_ctx, plan, h->ws + kHeaderBytes,
-                                       reinterpret_cast<int *>(h->ws + kCounterOffset), out, lse, out_anchor,
-                                       out_score, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = sla::launch_canary_fill(h->ws + kHeaderBytes, plan.canaries, st);
+    if (e == cudaSuccess)
+        e = sla::launch_decode(q_s, q, k_cache, v_cache, c, l->dtype, n_ctx, plan, h->ws + kHeaderBytes,
+                               reinterpret_cast<int *>(h->ws + kCounterOffset), out, lse, out_anchor, out_score, st);
+    if (e == cudaSuccess) e = sla::launch_canary_check(h->ws + kHeaderBytes, plan.canaries, c.status, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "sla_decode_step");
     h->launches += 2;
+    if (plan.canaries.n) { h->last_canaries = plan.canaries; h->last_canary_base = h->ws + kHeaderBytes; }
     return SLA_OK;
 }
 

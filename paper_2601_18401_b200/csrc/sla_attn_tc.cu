@@ -946,7 +946,7 @@ bool tc_attention_supported(const Call &c, int dtype) {
 }
 
 // Scratch layout for a chunk of Lc query positions; returns total bytes.
-TcPlan plan_attention_tc(const Call &c, int Lc) {
+TcPlan plan_attention_tc(const Call &c, int Lc, size_t gap) {
     TcPlan p;
     p.Lc = Lc;
     p.n_bg = c.B * c.Hkv;
@@ -1003,28 +1003,38 @@ TcPlan plan_attention_tc(const Call &c, int Lc) {
     // gaps between end blocks (fewer than NB per list)
     p.max_tiles = (long long)(slots / kRows) + (long long)p.n_bg * (p.NB + 1) + 1;
     size_t off = 0;
-    p.off_counters = off; off = align256(off + 64 + (size_t)p.n_bg * 8);
-    p.off_key_count = off; off = align256(off + n_keys * 4);
-    p.off_key_cursor = off; off = align256(off + n_keys * 4);
-    p.off_cta_hist = off; off = align256(off + (size_t)p.ctas_per_bg * n_keys * 4);
-    p.off_tiles = off; off = align256(off + (size_t)p.max_tiles * 16);
-    p.off_recs = off; off = align256(off + slots * 16);
-    p.off_npieces = off; off = align256(off + rows);
-    p.off_part_lse = off; off = align256(off + slots * 8);
-    p.off_part_o = off; off = align256(off + slots * kD * 2);
+    // a region of `size` bytes at the next 256-byte boundary, with a canary gap before it when asked for
+    auto take = [&](size_t size) {
+        if (gap) { p.canaries.add(off); off += gap; }
+        const size_t at = off;
+        off = align256(off + size);
+        return at;
+    };
+    p.off_counters = take(64 + (size_t)p.n_bg * 8);
+    // the two bucket tables are cleared together at the start of every chunk: no gap between them
+    p.off_key_count = take(2 * align256(n_keys * 4));
+    p.off_key_cursor = p.off_key_count + align256(n_keys * 4);
+    p.off_cta_hist = take((size_t)p.ctas_per_bg * n_keys * 4);
+    p.off_tiles = take((size_t)p.max_tiles * 16);
+    p.off_recs = take(slots * 16);
+    p.off_npieces = take(rows);
+    p.off_part_lse = take(slots * 8);
+    p.off_part_o = take(slots * kD * 2);
+    if (gap) { p.canaries.add(off); off += gap; }
     p.bytes = off;
     return p;
 }
 
 cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor,
                            const float *score, void *out, float *lse, float *lse_span, void *scratch, size_t scratch_bytes, int sm_count,
-                           cudaStream_t st, long long *launches, KernelTimer *timer) {
+                           cudaStream_t st, long long *launches, KernelTimer *timer, bool canaries) {
     // the largest chunk of query positions whose scratch fits
+    const size_t gap = canaries ? Canaries::kBytes : 0;
     long long Lc = c.Lq;
-    TcPlan plan = plan_attention_tc(c, (int)Lc);
+    TcPlan plan = plan_attention_tc(c, (int)Lc, gap);
     while (plan.bytes > scratch_bytes && Lc > 1) {
         Lc = (Lc + 1) / 2;
-        plan = plan_attention_tc(c, (int)Lc);
+        plan = plan_attention_tc(c, (int)Lc, gap);
     }
     if (plan.bytes > scratch_bytes || !plan.ok) return cudaErrorMemoryAllocation;
     if (plan.max_tiles > (1ll << 30) || (long long)c.B * c.Hq * Lc * plan.slots > (1ll << 31) - 1) return cudaErrorInvalidValue;
@@ -1046,8 +1056,9 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
     for (long long r0 = 0; r0 < c.Lq; r0 += Lc) {
         const int lc = (int)((c.Lq - r0 < Lc) ? c.Lq - r0 : Lc);
         const long long rows = (long long)c.B * c.Hq * lc;
-        cudaError_t e = cudaMemsetAsync(ws + plan.off_key_count, 0, plan.off_cta_hist - plan.off_key_count, st);
+        cudaError_t e = cudaMemsetAsync(ws + plan.off_key_count, 0, 2 * (plan.off_key_cursor - plan.off_key_count), st);
         if (e != cudaSuccess) return e;
+        if (canaries && (e = launch_canary_fill(ws, plan.canaries, st)) != cudaSuccess) return e;
         tc::PrepArgs pa;
         pa.anchor = anchor; pa.B = c.B; pa.Hq = c.Hq; pa.Hkv = c.Hkv; pa.G = c.G; pa.top_k = c.top_k;
         pa.span_len = c.span_len; pa.back = c.back; pa.fwd = c.fwd; pa.Lq = c.Lq; pa.q_pos0 = c.q_pos0;
@@ -1093,6 +1104,7 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         if (launches) *launches += 2;
+        if (canaries && (e = launch_canary_check(ws, plan.canaries, c.status, st)) != cudaSuccess) return e;
     }
     return cudaSuccess;
 }

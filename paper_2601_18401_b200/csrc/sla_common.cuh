@@ -10,7 +10,7 @@
 namespace sla {
 
 // Bits of the device status word (first int of the handle's workspace).
-enum : int { kStatusTimeout = 1, kStatusBadIndex = 2 };
+enum : int { kStatusTimeout = 1, kStatusBadIndex = 2, kStatusOverrun = 4 };
 
 constexpr int kMaxTopK = 64;
 constexpr int kMaxGroup = 16;

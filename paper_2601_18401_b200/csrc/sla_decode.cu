@@ -755,7 +755,7 @@ int decode_attn_blocks_per_sm(int dtype, int D) {
     return slot;
 }
 
-DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots) {
+DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots, size_t gap) {
     DecodePlan p;
     // candidates: the strides whose anchor lies left of the local window
     const long long n_cand = n_strides(c, n_ctx - 1) - window_strides(c);
@@ -773,13 +773,21 @@ DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots) {
     if (ns > 256) ns = 256;
     if (ns < 1) ns = 1;
     p.n_splits = (int)ns;
-    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
     const size_t bh = (size_t)c.B * c.Hq, n_units = bh * units;
-    p.off_scores = 0;
-    p.off_spans = align(p.off_scores + bh * (size_t)p.n_anchor * sizeof(float));
-    p.off_partial = align(p.off_spans + n_units * (size_t)(2 * pcap + 2) * sizeof(int));
-    p.off_unit_out = align(p.off_partial + n_units * (size_t)p.n_splits * (c.D + 2) * sizeof(float));
-    p.bytes = align(p.off_unit_out + (per_span ? n_units * (size_t)(c.D + 2) * sizeof(float) : 0));
+    size_t off = 0;
+    // a region of `size` bytes at the next 256-byte boundary, with a canary gap before it when asked for
+    auto take = [&](size_t size) {
+        if (gap) { p.canaries.add(off); off += gap; }
+        const size_t at = off;
+        off = (off + size + 255) & ~(size_t)255;
+        return at;
+    };
+    p.off_scores = take(bh * (size_t)p.n_anchor * sizeof(float));
+    p.off_spans = take(n_units * (size_t)(2 * pcap + 2) * sizeof(int));
+    p.off_partial = take(n_units * (size_t)p.n_splits * (c.D + 2) * sizeof(float));
+    p.off_unit_out = take(per_span ? n_units * (size_t)(c.D + 2) * sizeof(float) : 0);
+    if (gap) { p.canaries.add(off); off += gap; }
+    p.bytes = off;
     return p;
 }
 

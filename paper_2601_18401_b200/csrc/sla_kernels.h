@@ -22,6 +22,19 @@ struct KernelTimer {
     void end(cudaStream_t st) { if (enabled && used < kMaxPairs) { cudaEventRecord(ev[2 * used + 1], st); ++used; } }
 };
 
+// Debug canaries: with a gap of kBytes between the regions of a call's scratch memory (and before the
+// first and after the last), filled with a pattern before the kernels run and checked after them, a
+// kernel that writes outside its region is reported through the status word instead of going unnoticed.
+struct Canaries {
+    static constexpr int kMax = 16;
+    static constexpr size_t kBytes = 256;
+    size_t at[kMax] = {};   // byte offsets of the gaps from the scratch base
+    int n = 0;
+    void add(size_t off) { if (n < kMax) at[n++] = off; }
+};
+cudaError_t launch_canary_fill(void *scratch, const Canaries &cn, cudaStream_t st);
+cudaError_t launch_canary_check(const void *scratch, const Canaries &cn, int *status, cudaStream_t st);
+
 // ---- tensor-core span-search for bf16 / head_dim 128 (sla_search_mma.cu) -------------------------
 bool search_mma_supported(const Call &c, int dtype);
 cudaError_t launch_search_mma(const void *q_s, const void *k, const Call &c, int32_t *out_anchor, float *out_score,
@@ -42,15 +55,16 @@ struct TcPlan {
     long long max_tiles;
     size_t off_counters, off_key_count, off_key_cursor, off_cta_hist, off_tiles, off_recs, off_npieces, off_part_lse,
         off_part_o, bytes;
+    Canaries canaries;
 };
 bool tc_attention_shape_ok(const Call &c, int dtype);  // host-only shape test
 bool tc_attention_supported(const Call &c, int dtype); // shape test + driver entry point present
-TcPlan plan_attention_tc(const Call &c, int Lc);
+TcPlan plan_attention_tc(const Call &c, int Lc, size_t gap = 0);   // gap: bytes of canary between regions
 // Splits the query rows into chunks whose scratch fits `scratch_bytes`; adds its kernel launches to
 // *launches.  Returns cudaErrorMemoryAllocation when not even one query position fits.
 cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor, const float *score,
                            void *out, float *lse, float *lse_span, void *scratch, size_t scratch_bytes, int sm_count,
-                           cudaStream_t st, long long *launches, KernelTimer *timer);
+                           cudaStream_t st, long long *launches, KernelTimer *timer, bool canaries = false);
 
 // ---- decode step (sla_decode.cu) ---------------------------------------------------------------
 // Scratch layout of one decode step, all offsets in bytes from the scratch base.
@@ -64,9 +78,10 @@ struct DecodePlan {
     size_t off_partial; // float [units][n_splits][D + 2]: running max, denominator, numerator
     size_t off_unit_out; // float [units][D + 2] (per-span mode): log-sum-exp and output of every unit
     size_t bytes;
+    Canaries canaries;
 };
 // cta_slots = SM count x resident decode_attn CTAs per SM (see decode_attn_blocks_per_sm)
-DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots);
+DecodePlan plan_decode(const Call &c, long long n_ctx, int cta_slots, size_t gap = 0);
 int decode_attn_blocks_per_sm(int dtype, int D);
 // counters: B*Hkv + B*Hq*units + B*Hq ints (units = top_k in the per-span mode, else 1), zero on entry
 // and zero again on exit (completion counters)
@@ -86,6 +101,10 @@ cudaError_t launch_decode_shard_attend(const void *q, const void *k_local, const
                                        float *partial_out, cudaStream_t st);
 cudaError_t launch_decode_shard_merge(const float *all_partial, int n_shards, const Call &c, int dtype, void *out,
                                       float *lse, cudaStream_t st);
+
+// ---- diagnostics (sla_diag.cu)
+cudaError_t launch_probe_l2_read(const void *buf, size_t bytes, int iters, int n_ctas, unsigned *sink, cudaStream_t st);
+cudaError_t launch_selftest_wait_expiry(int max_polls, int *status, int *polls_done, cudaStream_t st);
 
 // argument checks of a decode step without a handle (defined in sla_api.cu)
 sla_status_t check_decode_args(const void *q_s, const void *q, const void *k_cache, const void *v_cache,

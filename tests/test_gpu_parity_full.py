@@ -46,6 +46,7 @@ def run_prefill_config(sla, w, seed, rows, search_all_rows_heads=None):
     params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim)
     layout = sla.make_layout(x["q"], x["k"])
     handle = sla.Handle(0, sla.sla_workspace_bytes(layout, params, w.seq_len, w.seq_len) + (64 << 20))
+    sla.sla_set_debug_canaries(handle, True)
     anchor, score = sla.sla_span_search(handle, x["q_s"], x["k"], params)
     torch.cuda.synchronize()
     host = P.host_inputs(x)

@@ -20,6 +20,7 @@ def sla():
 @pytest.fixture(scope="module")
 def handle(sla):
     h = sla.Handle(0, 256 << 20)
+    sla.sla_set_debug_canaries(h, True)   # every attention and decode call of this module is checked for overruns
     yield h
     h.close()
 

@@ -19,6 +19,7 @@ def sla():
 @pytest.fixture(scope="module")
 def handle(sla):
     h = sla.Handle(0, 1 << 30)
+    sla.sla_set_debug_canaries(h, True)   # every attention and decode call of this module is checked for overruns
     yield h
     h.close()
 
@@ -242,6 +243,35 @@ def test_decode_parity(sla, handle, dtype, D, Hq, Hkv):
         torch.cuda.synchronize()
         P.check_decode_step(got, synth.to_numpy(step["q_s"]), synth.to_numpy(step["q"]), hk, hv, code, dtype,
                             n_ctx=n_ctx, top_k=top_k, span_len=span_len)
+
+
+def test_bounded_wait_expiry_is_reported_and_survivable(sla, handle):
+    """A device-side wait that runs out (a barrier nothing arrives on, a bounded number of polls) leaves the
+    time-out bit in the status word and returns by itself; the handle reports it once and keeps working."""
+    polls = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sla.sla_selftest_wait_expiry(handle, 1500, polls)
+    assert sla.sla_poll_status(handle) == -5          # SLA_ERR_DEVICE_TIMEOUT
+    assert int(polls.item()) == 1500
+    assert sla.sla_poll_status(handle) == sla.SLA_OK   # reported once
+    run_prefill(sla, handle, workload(n_q_heads=8, n_kv_heads=2, seq_len=900))
+    with pytest.raises(sla.SlaError):
+        sla.sla_selftest_wait_expiry(handle, 10 ** 6)
+
+
+def test_canaries_report_a_damaged_gap(sla, handle):
+    """The debug canaries between the scratch regions: intact after an ordinary decode step; once one word
+    of a gap is overwritten (by the self-test's own 4-byte memset) the check reports an overrun."""
+    from paper_2601_18401_b200 import synth
+    w = synth.Workload("c", "decode", 1, 8, 2, 128, 5000, "bf16", 40, 4, seed=3)
+    kc, vc = synth.make_decode_cache(w, "cuda:0", capacity=5000)
+    x = synth.make_decode_step_inputs(w, 0, "cuda:0")
+    sla.sla_decode_step(handle, x["q_s"], x["q"], kc, vc, 5000, sla.make_params(4, 40))
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    sla.sla_selftest_canary_trip(handle)
+    assert sla.sla_poll_status(handle) == -7           # SLA_ERR_DEVICE_OVERRUN
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
+    sla.sla_decode_step(handle, x["q_s"], x["q"], kc, vc, 5000, sla.make_params(4, 40))
+    assert sla.sla_poll_status(handle) == sla.SLA_OK
 
 
 def test_error_returns(sla, handle):
