@@ -37,11 +37,63 @@ from paper_2601_18401_b200 import synth
 METRIC = "prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one tc_attend launch of the default workload
-# (L = 65536), from the one-pass ncu capture of the full-size launch summarised in profiles/
+# (L = 65536): a CONSTANT taken from the one-pass ncu capture of the full-size launch summarised in
+# profiles/bench_prefill_L65536_launch_list.md, not something this run measures
 TC_ATTEND_DRAM_BYTES_PER_LAUNCH = {65536: 4.74e9, 16384: 0.887e9}
+TRAFFIC_SOURCE = "constant from the one-pass ncu capture summarised under profiles/, not measured by this run"
+NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16, per GPU
 # the same for one decode_attn launch (the dominant kernel of a decode step), by workload
 DECODE_ATTN_DRAM_BYTES_PER_LAUNCH = {"decode_1M": 485.2e6, "decode_10M": 1571.4e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def tensor_roofline(flops, kern_ms, region_s, clocks, peaks):
+    """Roofline entry of a tensor-core kernel.  The denominator is the measured burst rate of a bf16
+    matmul when the timed region is short (under a second) or the sampled SM clock stayed at 95 % of
+    its maximum or more -- the conditions under which the burst figure was measured -- and the
+    sustained rate (measured over seconds under the power cap) otherwise; both fractions and the one
+    of the nominal dense peak are given beside it."""
+    tflops = flops / (kern_ms * 1e-3) / 1e12
+    burst, sustained = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    at_full_clock = bool(mhz and mx and mhz >= 0.95 * mx)
+    use_burst = region_s < 1.0 or at_full_clock
+    peak = burst if use_burst else sustained
+    return {"bound": "tensor", "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
+            "frac_of_burst": tflops / burst, "frac_of_sustained": tflops / sustained,
+            "frac_of_nominal": tflops / NOMINAL_BF16_TFLOPS, "nominal_peak": NOMINAL_BF16_TFLOPS,
+            "peak_rule": ("burst" if use_burst else "sustained") + f": timed region {region_s:.2f} s, median SM clock "
+                         f"{mhz} of {mx} MHz",
+            "ms_times_sm_mhz": (kern_ms * mhz) if mhz else None,
+            "flops_per_launch": flops, "ms_per_launch": kern_ms, "peak_source": peaks["_source"]}
+
+
+def search_key_bytes(B, Hkv, L, D, elem, window=0):
+    """Algorithmic bytes of the span-search kernel's dominant stream: one key row per (position, stride,
+    KV head) -- sum over i of the number of candidate strides floor(sqrt(i+1)) - floor(sqrt(w))."""
+    i = np.arange(1, L + 1, dtype=np.float64)
+    n = np.floor(np.sqrt(i)).astype(np.int64)
+    n = np.where((n * n > i), n - 1, n)
+    n = np.where(((n + 1) * (n + 1) <= i), n + 1, n)
+    n = np.maximum(n - int(np.floor(np.sqrt(window))), 0)
+    return int(n.sum()) * B * Hkv * D * elem
+
+
+def measure_l2_probe(sla, handle, dev, mib=32, iters=2, reps=5):
+    """GB/s of the library's read-only L2 probe over an L2-resident buffer."""
+    buf = torch.empty(mib << 20, dtype=torch.uint8, device=dev).zero_()
+    for _ in range(3):
+        nbytes = sla.sla_probe_l2_read(handle, buf, iters)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        sla.sla_probe_l2_read(handle, buf, iters)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    return {"gbs": nbytes / (ms * 1e-3) / 1e9, "buffer_mib": mib, "bytes_per_launch": nbytes, "ms_per_launch": ms,
+            "how": "every CTA of a 4 x SM-count grid reads the whole buffer with 32-byte loads"}
 
 
 def load_peaks():
@@ -176,7 +228,34 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def bench_decode(sla, handle, w, steps, peaks, dev):
+def oracle_decode_us(w, kc, vc, x, n_ctx):
+    """The CPU oracle's decode step on the same cache and inputs, timed on the host cores.  The host
+    copy of the cache is sparse -- only the rows the step reads (its anchor rows, then the spans of the
+    anchors the oracle itself selects) are fetched; the rest of the (virtual) array is never touched."""
+    from oracle import sla_oracle as O
+    shape = tuple(kc.shape)
+    hk, hv = np.empty(shape, dtype=np.uint16), np.empty(shape, dtype=np.uint16)
+    i = n_ctx - 1
+    m = np.arange(1, int(np.floor(np.sqrt(i + 1))) + 2, dtype=np.int64)
+    t = i + 1 - m * m
+    t = torch.from_numpy(t[t >= 0]).to(kc.device)
+    hk[:, :, t.cpu().numpy()] = synth.to_numpy(kc[:, :, t])
+    q_s, q = synth.to_numpy(x["q_s"]), synth.to_numpy(x["q"])
+    code = synth.dtype_code(w.dtype)
+    sel = O.span_search(q_s[:, :, None], hk, code, top_k=w.top_k, q_pos0=i, Lkv=n_ctx)["anchor"]
+    span = w.back_factor * w.span_len
+    for tpos in np.unique(sel[sel >= 0]):
+        lo, hi = max(0, int(tpos) - span), min(i, int(tpos) + w.fwd_factor * w.span_len)
+        hk[:, :, lo:hi + 1] = synth.to_numpy(kc[:, :, lo:hi + 1])
+        hv[:, :, lo:hi + 1] = synth.to_numpy(vc[:, :, lo:hi + 1])
+    t0 = time.perf_counter()
+    O.decode_step(q_s, q, hk, hv, code, n_ctx=n_ctx, top_k=w.top_k, span_len=w.span_len,
+                  back_factor=w.back_factor, fwd_factor=w.fwd_factor)
+    return {"value": (time.perf_counter() - t0) * 1e6, "unit": "us per decode step", "cores": O.threads(), "kind": "oracle",
+            "sample": "one whole decode step (search over all anchors + attention over the selected spans)"}
+
+
+def bench_decode(sla, handle, w, steps, peaks, dev, with_oracle=False):
     """Decode loop: append the new token's K/V, then one sla_decode_step, `steps` times."""
     kc, vc = synth.make_decode_cache(w, dev, capacity=w.seq_len + steps + 8)
     params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim)
@@ -223,13 +302,15 @@ def bench_decode(sla, handle, w, steps, peaks, dev):
     n_anchor = int(np.floor(np.sqrt(w.seq_len + steps)))
     bytes_step = pairs * 2 * w.head_dim * elem + n_anchor * w.batch * w.n_kv_heads * w.head_dim * elem
     gbs = bytes_step / (us_call * 1e-6) / 1e9
+    cpu = oracle_decode_us(w, kc, vc, ins[(steps - 1) % len(ins)], w.seq_len + steps) if with_oracle else None
     del kc, vc
     torch.cuda.empty_cache()
     return {"workload": w.name, "us_per_token_per_layer": us, "us_per_decode_call": us_call, "steps": steps,
-            "algorithmic_bytes_per_step": bytes_step,
+            "algorithmic_bytes_per_step": bytes_step, "cpu_baseline": cpu,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0,
-                         "traffic": DECODE_ATTN_DRAM_BYTES_PER_LAUNCH.get(w.name), "peak_source": peaks["_source"]}}
+                         "traffic": DECODE_ATTN_DRAM_BYTES_PER_LAUNCH.get(w.name), "traffic_source": TRAFFIC_SOURCE,
+                         "peak_source": peaks["_source"]}}
 
 
 def max_over_ranks(value: float, dist, device) -> float:
@@ -304,6 +385,84 @@ def measure_e2e(sla, handle, host, params, args, dist, dev, world, B, L):
             "ms_per_step": e2e_s * 1e3}
 
 
+def measure_prefill(sla, handle, w, x, steps, warmup, local, dist, dev, peaks):
+    """Times `steps` prefill steps (sla_span_search + sla_span_attention over the whole batch) with CUDA
+    events on the launching stream; returns the timings, the clocks sampled meanwhile, the launches
+    counted, the roofline of the attention kernel and that of the search kernel."""
+    B, Hq, L, D = x["q"].shape
+    params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim)
+    anchor = torch.empty(B, Hq, L, w.top_k, dtype=torch.int32, device=dev)
+    score = torch.empty(B, Hq, L, w.top_k, dtype=torch.float32, device=dev)
+    out = torch.empty_like(x["q"])
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
+
+    def step(ev=None):
+        sla.sla_span_search(handle, x["q_s"], x["k"], params, out_anchor=anchor, out_score=score)
+        if ev is not None:
+            ev[0].record()
+        sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params, out=out, lse=lse)
+        if ev is not None:
+            ev[1].record()
+
+    for _ in range(max(3, warmup)):
+        step()
+    torch.cuda.synchronize()
+    sla.sla_set_kernel_timing(handle, True)   # events around the main attention kernel, on its stream
+    launches0 = sla.sla_kernel_launches(handle)
+    sampler = ClockSampler(local)
+    sampler.start()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for s in range(steps):
+        step(evs[s])
+    t1.record()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    clocks = sampler.stop()
+    launches = sla.sla_kernel_launches(handle) - launches0
+    total_ms = t0.elapsed_time(t1)
+    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    kern_ms_sum, kern_n = sla.sla_kernel_time_ms(handle)
+    sla.sla_set_kernel_timing(handle, False)
+    kern_ms = kern_ms_sum / steps if kern_n else attn_ms   # generic path: whole call
+    total_ms = max_over_ranks(total_ms, dist, dev)
+    ms_per_step = total_ms / steps
+    search_ms = ms_per_step - attn_ms
+
+    # roofline of the dominant kernel (span-attention): 4*D flops per attended (query, key) pair
+    pairs = attended_pairs(anchor, w.span_len, w.back_factor, w.fwd_factor)
+    flops = 4.0 * D * pairs
+    roofline = tensor_roofline(flops, kern_ms, total_ms * 1e-3, clocks, peaks)
+    roofline["kernel"] = "tc_attend (tcgen05 span-attention)" if kern_n else "attn_rows_simt"
+    roofline["launches_timed"] = kern_n
+    roofline["traffic"] = TC_ATTEND_DRAM_BYTES_PER_LAUNCH.get(L) if (kern_n and w.name.startswith("prefill_L65536")) else None
+    roofline["traffic_source"] = TRAFFIC_SOURCE if roofline["traffic"] else None
+    roofline["whole_call"] = {"sla_span_attention_ms": attn_ms, "sla_span_search_ms": search_ms,
+                              "attention_tflops": flops / (attn_ms * 1e-3) / 1e12,
+                              "attention_frac_of_burst": flops / (attn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                              "attention_frac_of_sustained": flops / (attn_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]}
+    del anchor, score, out, lse
+    return {"ms_per_step": ms_per_step, "attn_ms": attn_ms, "search_ms": search_ms, "kern_ms": kern_ms,
+            "clocks": clocks, "launches": int(launches), "roofline": roofline, "params": params}
+
+
+def search_roofline(w, search_ms, probe):
+    """The span-search kernel streams one key row per (position, stride, KV head) out of L2 (K is
+    L2-resident per KV head); its roofline is the L2 read bandwidth the probe measured in this run."""
+    elem = 2 if w.dtype == "bf16" else 4
+    nbytes = search_key_bytes(w.batch, w.n_kv_heads, w.seq_len, w.head_dim, elem, w.window)
+    gbs = nbytes / (search_ms * 1e-3) / 1e9
+    return {"bound": "l2", "kernel": "search_diag (span-search, selection folded into the scoring loop)",
+            "achieved": gbs, "peak": probe["gbs"], "unit": "GB/s", "frac": gbs / probe["gbs"],
+            "algorithmic_bytes_per_launch": nbytes, "ms_per_launch": search_ms, "traffic": None,
+            "peak_source": f"read-only L2 probe of this run ({probe['buffer_mib']} MiB buffer, {probe['how']})"}
+
+
 def run_ours(args, w):
     import paper_2601_18401_b200 as sla
     rank = int(os.environ.get("RANK", "0"))
@@ -329,62 +488,9 @@ def run_ours(args, w):
     stage = sla.sla_host_staging_bytes(layout, params, w.seq_len)
     handle = sla.Handle(local, work + stage + (64 << 20))
     B, Hq, L, D = x["q"].shape
-    anchor = torch.empty(B, Hq, L, w.top_k, dtype=torch.int32, device=dev)
-    score = torch.empty(B, Hq, L, w.top_k, dtype=torch.float32, device=dev)
-    out = torch.empty_like(x["q"])
-    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
-
-    def step(ev=None):
-        sla.sla_span_search(handle, x["q_s"], x["k"], params, out_anchor=anchor, out_score=score)
-        if ev is not None:
-            ev[0].record()
-        sla.sla_span_attention(handle, x["q"], x["k"], x["v"], anchor, params, out=out, lse=lse)
-        if ev is not None:
-            ev[1].record()
-
-    for _ in range(max(3, args.warmup)):
-        step()
-    torch.cuda.synchronize()
-    sla.sla_set_kernel_timing(handle, True)   # events around the main attention kernel, on its stream
-    launches0 = sla.sla_kernel_launches(handle)
-    sampler = ClockSampler(local)
-    sampler.start()
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for s in range(args.steps):
-        step(evs[s])
-    t1.record()
-    torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
-    clocks = sampler.stop()
-    launches = sla.sla_kernel_launches(handle) - launches0
-    total_ms = t0.elapsed_time(t1)
-    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
-    kern_ms_sum, kern_n = sla.sla_kernel_time_ms(handle)
-    sla.sla_set_kernel_timing(handle, False)
-    kern_ms = kern_ms_sum / args.steps if kern_n else attn_ms   # generic path: whole call
-    total_ms = max_over_ranks(total_ms, dist, dev)
-    ms_per_step = total_ms / args.steps
-    value = world * B * L / (ms_per_step * 1e-3)
-
-    # roofline of the dominant kernel (span-attention): 4*D flops per attended (query, key) pair
-    pairs = attended_pairs(anchor, w.span_len, w.back_factor, w.fwd_factor)
-    flops = 4.0 * D * pairs
-    tflops = flops / (kern_ms * 1e-3) / 1e12
-    peak_tf = peaks["bf16_tflops_sustained"]
-    roofline = {"bound": "tensor", "kernel": "tc_attend (tcgen05 span-attention)" if kern_n else "attn_rows_simt",
-                "achieved": tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": tflops / peak_tf,
-                "traffic": TC_ATTEND_DRAM_BYTES_PER_LAUNCH.get(L) if kern_n else None,
-                "flops_per_launch": flops, "ms_per_launch": kern_ms, "launches_timed": kern_n,
-                "whole_call": {"sla_span_attention_ms": attn_ms, "sla_span_search_ms": ms_per_step - attn_ms,
-                               "attention_tflops": flops / (attn_ms * 1e-3) / 1e12,
-                               "attention_frac": flops / (attn_ms * 1e-3) / 1e12 / peak_tf},
-                "peak_source": peaks["_source"] + " (sustained bf16 matmul; the kernel runs inside a long step)"}
+    m = measure_prefill(sla, handle, w, x, args.steps, args.warmup, local, dist, dev, peaks)
+    value = world * B * L / (m["ms_per_step"] * 1e-3)
+    probe = measure_l2_probe(sla, handle, dev)
 
     # end to end through the host-buffer C call: pinned host inputs, host outputs, copies inside
     host = None
@@ -394,44 +500,72 @@ def run_ours(args, w):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": max(3, args.warmup), "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "batch_per_gpu": B, "q_heads": Hq, "kv_heads": w.n_kv_heads, "head_dim": D,
                    "seq_len": L, "span_len": w.span_len, "top_k": w.top_k, "back_factor": w.back_factor,
                    "fwd_factor": w.fwd_factor, "planted_spans": w.planted_spans,
                    "l2": "inputs (1.3 GB) exceed the 126 MB L2; no flush between steps",
                    "parallelism": f"independent sequences x{world}"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+        "clocks": m["clocks"], "e2e": e2e, "gpu_launches": m["launches"], "roofline": m["roofline"],
+        "roofline_search": search_roofline(w, m["search_ms"], probe), "l2_probe": probe,
     }
 
     if rank == 0 and not args.no_decode and not args.seq_len:
         line["paper_kernel_config"] = bench_paper_config(sla, handle, dev, max(3, min(args.steps, 10)))
+    cpu_rows = None
+    if rank == 0 and not args.no_cpu_baseline:
+        cpu_rows = oracle_sample_rows(L, args.ref_rows)
+        cpu_rows = cpu_rows[cpu_rows < L]
+        cpu_host = {n: synth.to_numpy(t) for n, t in host.items()}
+    del x
+    handle.close()
+    torch.cuda.empty_cache()
+    if rank == 0 and not args.no_decode and not args.seq_len and not args.no_stress:
+        line["prefill_stress_L262144"] = bench_stress(sla, local, dev, peaks, probe, max(3, min(args.steps, 5)))
     if rank == 0 and not args.no_decode:
-        del x, anchor, score, out, lse
-        torch.cuda.empty_cache()
+        dh = sla.Handle(local, 64 << 20)
         dec = []
         for ci, steps in ((3, 256), (4, 128)):
             if args.decode_only and args.decode_only != synth.CONFIGS[ci].name:
                 continue
             try:
-                dec.append(bench_decode(sla, handle, synth.CONFIGS[ci], steps if not args.quick else 16, peaks, dev))
+                dec.append(bench_decode(sla, dh, synth.CONFIGS[ci], steps if not args.quick else 16, peaks, dev,
+                                        with_oracle=not args.no_cpu_baseline))
             except torch.cuda.OutOfMemoryError as e:  # pragma: no cover
                 dec.append({"workload": synth.CONFIGS[ci].name, "skipped": f"out of memory: {e}"})
         line["decode"] = dec
-    if rank == 0 and not args.no_cpu_baseline:
+        dh.close()
+    if cpu_rows is not None:
         from oracle import sla_oracle as O
-        rows = oracle_sample_rows(L, args.ref_rows)
-        hn = {n: synth.to_numpy(t) for n, t in host.items()}
-        rows = rows[rows < L]
-        secs = time_oracle_prefill(w, hn, rows)
-        line["cpu_baseline"] = {"value": len(rows) * B / secs, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
-                                "sample": f"{len(rows)} evenly spaced query positions x all {Hq} heads, "
+        secs = time_oracle_prefill(w, cpu_host, cpu_rows)
+        line["cpu_baseline"] = {"value": len(cpu_rows) * B / secs, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
+                                "sample": f"{len(cpu_rows)} evenly spaced query positions x all {Hq} heads, "
                                           f"search + attention, {secs:.1f} s"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def bench_stress(sla, local, dev, peaks, probe, steps):
+    """The largest prefill configuration (batch 2, 16/4 heads, L = 262144, l = 512, k = 16): the same step,
+    timed the same way, reported beside the headline."""
+    w = synth.CONFIGS[2]
+    x = synth.make_prefill(w, device=dev)
+    params = sla.make_params(w.top_k, w.span_len, w.back_factor, w.fwd_factor, head_dim=w.head_dim)
+    layout = sla.make_layout(x["q"], x["k"])
+    handle = sla.Handle(local, sla.sla_workspace_bytes(layout, params, w.seq_len, w.seq_len) + (64 << 20))
+    m = measure_prefill(sla, handle, w, x, steps, 3, local, None, dev, peaks)
+    B, Hq, L, D = x["q"].shape
+    del x
+    handle.close()
+    torch.cuda.empty_cache()
+    return {"workload": w.name, "batch": B, "q_heads": Hq, "kv_heads": w.n_kv_heads, "seq_len": L, "span_len": w.span_len,
+            "top_k": w.top_k, "steps": steps, "ms_per_step": m["ms_per_step"], "tokens_per_s": B * L / (m["ms_per_step"] * 1e-3),
+            "clocks": m["clocks"], "gpu_launches": m["launches"], "roofline": m["roofline"],
+            "roofline_search": search_roofline(w, m["search_ms"], probe)}
 
 
 def main():
@@ -447,6 +581,7 @@ def main():
     ap.add_argument("--seq-len", type=int, default=0, help="shorter prefill sequence (for profiler captures)")
     ap.add_argument("--decode-only", default="", help="decode_1M or decode_10M: only that decode loop besides the prefill part")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-stress", action="store_true", help="skip the L = 262144 configuration reported beside the headline")
     ap.add_argument("--quick", action="store_true", help="short decode loops (for smoke runs)")
     args = ap.parse_args()
     w = synth.CONFIGS[args.workload]
