@@ -19,12 +19,18 @@ def shard_range(cache_len: int, rank: int, world: int) -> tuple[int, int]:
 
 
 def _gather(t: torch.Tensor, group) -> torch.Tensor:
-    """All ranks' copies of `t`, stacked in rank order: [world, ...]."""
+    """All ranks' copies of `t`, stacked in rank order: [world, ...].  With a backend that has no device
+    collectives (gloo) a device tensor is staged through the host."""
     import torch.distributed as dist
     world = dist.get_world_size(group)
-    parts = [torch.empty_like(t) for _ in range(world)]
-    dist.all_gather(parts, t.contiguous(), group=group)
-    return torch.stack(parts)
+    src = t.contiguous()
+    staged = src.is_cuda and dist.get_backend(group) == "gloo"
+    if staged:
+        src = src.cpu()
+    parts = [torch.empty_like(src) for _ in range(world)]
+    dist.all_gather(parts, src, group=group)
+    out = torch.stack(parts)
+    return out.to(t.device) if staged else out
 
 
 def decode_step_sharded(handle: B.Handle, q_s: torch.Tensor, q: torch.Tensor, k_local: torch.Tensor,
