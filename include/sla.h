@@ -149,6 +149,14 @@ int64_t sla_kernel_launches(sla_handle_t handle);
 sla_status_t sla_set_kernel_timing(sla_handle_t handle, int enable);
 sla_status_t sla_kernel_time_ms(sla_handle_t handle, float *ms, int32_t *n_launches);
 
+/* Work statistics of the most recent tensor-core span-attention call of this handle (its last chunk of
+ * query positions); a diagnostic for benchmarks, the paper has no counterpart.  out4_host (host memory)
+ * receives: tiles of up to 128 pieces, pieces, the sum over tiles of 64-key blocks walked, and the sum
+ * over pieces of the blocks their tile walked.  128 x 64 x (third value) is the number of (row, key)
+ * products the tensor cores executed, against which the attended pairs measure how well the tiles were
+ * packed.  Waits for `stream`. */
+sla_status_t sla_attention_tile_stats(sla_handle_t handle, int64_t *out4_host, void *stream);
+
 /* Debug canaries (the paper has no counterpart; they stand in for a memory checker).  When enabled,
  * sla_span_attention, sla_span_attention_gated and sla_decode_step separate the regions of their scratch
  * memory by 256-byte gaps, fill the gaps with a pattern before their kernels run and check them

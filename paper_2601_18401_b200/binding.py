@@ -28,7 +28,7 @@ EXPORTS = [
     "sla_kernel_time_ms", "sla_decode_step_static", "sla_span_attention_gated",
     "sla_decode_shard_search", "sla_decode_shard_attend", "sla_decode_shard_merge",
     "sla_pattern_offsets", "sla_pattern_len_steps", "sla_probe_l2_read", "sla_selftest_wait_expiry",
-    "sla_set_debug_canaries", "sla_selftest_canary_trip",
+    "sla_set_debug_canaries", "sla_selftest_canary_trip", "sla_attention_tile_stats",
 ]
 
 
@@ -105,6 +105,8 @@ def load_library():
     lib.sla_host_staging_bytes.argtypes = [LP, PP, i64]
     lib.sla_prefill_host.restype = i32
     lib.sla_prefill_host.argtypes = [vp, vp, vp, vp, vp, i64, LP, PP, vp, vp, vp, vp, vp]
+    lib.sla_attention_tile_stats.restype = i32
+    lib.sla_attention_tile_stats.argtypes = [vp, vp, vp]
     lib.sla_set_debug_canaries.restype = i32
     lib.sla_set_debug_canaries.argtypes = [vp, i32]
     lib.sla_selftest_canary_trip.restype = i32
@@ -230,6 +232,13 @@ def sla_kernel_time_ms(handle: Handle):
     ms, n = C.c_float(0.0), C.c_int32(0)
     handle.check(handle._lib.sla_kernel_time_ms(handle.ptr, C.byref(ms), C.byref(n)), "sla_kernel_time_ms")
     return float(ms.value), int(n.value)
+
+
+def sla_attention_tile_stats(handle: Handle, stream=None) -> dict:
+    """Tiles, pieces and key blocks walked by the most recent tensor-core span-attention call (last chunk)."""
+    buf = (C.c_int64 * 4)()
+    handle.check(handle._lib.sla_attention_tile_stats(handle.ptr, buf, _stream_ptr(stream)), "sla_attention_tile_stats")
+    return {"tiles": int(buf[0]), "pieces": int(buf[1]), "tile_blocks": int(buf[2]), "piece_blocks": int(buf[3])}
 
 
 def sla_set_debug_canaries(handle: Handle, enable: bool) -> None:

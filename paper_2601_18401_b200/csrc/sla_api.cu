@@ -18,6 +18,7 @@ struct sla_handle_s {
     long long launches = 0;   // kernels launched through this handle
     size_t scratch_avail = 0; // bytes of workspace after the header that kernels may use as scratch
     sla::KernelTimer timer;   // sla_set_kernel_timing / sla_kernel_time_ms
+    sla::TcLast tc_last;      // tile table of the most recent tensor-core attention chunk
     bool canaries = false;    // sla_set_debug_canaries
     sla::Canaries last_canaries;   // of the most recent call that laid any, and where its scratch began
     char *last_canary_base = nullptr;
@@ -288,6 +289,20 @@ int32_t sla_pattern_len_steps(double p, int64_t reach, int32_t *out, int32_t cap
     return (int32_t)t.size();
 }
 
+sla_status_t sla_attention_tile_stats(sla_handle_t h, int64_t *out4_host, void *stream) {
+    if (!h || !out4_host) return SLA_ERR_INVALID_ARG;
+    if (!h->tc_last.tiles) return fail(h, SLA_ERR_INVALID_ARG, "no tensor-core span-attention has run on this handle%s");
+    if (const char *why = check_device(h)) return fail(h, SLA_ERR_INVALID_ARG, "%s", why);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // four counters in the status header's spare space (bytes 64..95 of the workspace)
+    long long *dev = reinterpret_cast<long long *>(h->ws + 64);
+    cudaError_t e = sla::launch_tile_stats(h->tc_last, dev, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out4_host, dev, 4 * sizeof(long long), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "sla_attention_tile_stats");
+    return SLA_OK;
+}
+
 sla_status_t sla_set_debug_canaries(sla_handle_t h, int enable) {
     if (!h) return SLA_ERR_INVALID_ARG;
     h->canaries = enable != 0;
@@ -471,7 +486,7 @@ sla_status_t span_attention_impl(sla_handle_t h, const void *q, const void *k, c
             if (probe.bytes > h->scratch_avail)
                 return fail(h, SLA_ERR_WORKSPACE, "workspace too small for span-attention: ask sla_workspace_bytes%s");
             cudaError_t e = sla::launch_attn_tc(q, k, v, c, anchor, score, out, lse, lse_span, h->ws + kHeaderBytes,
-                                                h->scratch_avail, h->sm_count, st, &h->launches, &h->timer, h->canaries);
+                                                h->scratch_avail, h->sm_count, st, &h->launches, &h->timer, h->canaries, &h->tc_last);
             if (e != cudaSuccess) return cuda_fail(h, e, what);
             return SLA_OK;
         }

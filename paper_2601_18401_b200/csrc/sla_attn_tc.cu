@@ -928,7 +928,27 @@ bool make_kv_map(CUtensorMap *tm, const void *ptr, const Call &c, int slot[3]) {
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// out[0] tiles, out[1] pieces, out[2] sum over tiles of (key blocks walked), out[3] sum of pieces x blocks
+__global__ void __launch_bounds__(256) tile_stats(const int4 *__restrict__ tiles, const int *__restrict__ n_tiles,
+                                                  unsigned long long *out) {
+    const int n = *n_tiles;
+    unsigned long long a = 0, b = 0, c2 = 0;
+    for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < n; t += gridDim.x * blockDim.x) {
+        const int w = tiles[t].w, cnt = w & 0xff, nblk = w >> 8;
+        a += cnt; b += nblk; c2 += (unsigned long long)cnt * nblk;
+    }
+    atomicAdd(out + 1, a); atomicAdd(out + 2, b); atomicAdd(out + 3, c2);
+    if (blockIdx.x == 0 && threadIdx.x == 0) out[0] = n;
+}
+
 }  // namespace
+
+cudaError_t launch_tile_stats(const TcLast &last, long long *out4_device, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(out4_device, 0, 4 * sizeof(long long), st);
+    if (e != cudaSuccess) return e;
+    tile_stats<<<64, 256, 0, st>>>(last.tiles, last.n_tiles, reinterpret_cast<unsigned long long *>(out4_device));
+    return cudaGetLastError();
+}
 
 bool tc_attention_shape_ok(const Call &c, int dtype) {
     if (dtype != SLA_BF16 || c.D != kD) return false;
@@ -1027,7 +1047,7 @@ TcPlan plan_attention_tc(const Call &c, int Lc, size_t gap) {
 
 cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor,
                            const float *score, void *out, float *lse, float *lse_span, void *scratch, size_t scratch_bytes, int sm_count,
-                           cudaStream_t st, long long *launches, KernelTimer *timer, bool canaries) {
+                           cudaStream_t st, long long *launches, KernelTimer *timer, bool canaries, TcLast *last) {
     // the largest chunk of query positions whose scratch fits
     const size_t gap = canaries ? Canaries::kBytes : 0;
     long long Lc = c.Lq;
@@ -1089,6 +1109,7 @@ cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Ca
         tp.n_tiles = counters;
         tp.part_o = (__half *)(ws + plan.off_part_o); tp.part_lse = (float2 *)(ws + plan.off_part_lse);
         tp.status = c.status; tp.Hkv = c.Hkv;
+        if (last) { last->tiles = pa.tiles; last->n_tiles = counters; }
         if (timer) timer->begin(st);
         tc_attend<<<2 * sm_count, kThreads, kSmemBytes, st>>>(tm_k, tm_v, tp);
         if (timer) timer->end(st);

@@ -60,11 +60,15 @@ struct TcPlan {
 bool tc_attention_shape_ok(const Call &c, int dtype);  // host-only shape test
 bool tc_attention_supported(const Call &c, int dtype); // shape test + driver entry point present
 TcPlan plan_attention_tc(const Call &c, int Lc, size_t gap = 0);   // gap: bytes of canary between regions
+// Where the tile table of the most recent chunk lives (for sla_attention_tile_stats).
+struct TcLast { const int4 *tiles = nullptr; const int *n_tiles = nullptr; };
+cudaError_t launch_tile_stats(const TcLast &last, long long *out4_device, cudaStream_t st);
 // Splits the query rows into chunks whose scratch fits `scratch_bytes`; adds its kernel launches to
 // *launches.  Returns cudaErrorMemoryAllocation when not even one query position fits.
 cudaError_t launch_attn_tc(const void *q, const void *k, const void *v, const Call &c, const int32_t *anchor, const float *score,
                            void *out, float *lse, float *lse_span, void *scratch, size_t scratch_bytes, int sm_count,
-                           cudaStream_t st, long long *launches, KernelTimer *timer, bool canaries = false);
+                           cudaStream_t st, long long *launches, KernelTimer *timer, bool canaries = false,
+                           TcLast *last = nullptr);
 
 // ---- decode step (sla_decode.cu) ---------------------------------------------------------------
 // Scratch layout of one decode step, all offsets in bytes from the scratch base.

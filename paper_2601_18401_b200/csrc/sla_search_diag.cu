@@ -57,6 +57,12 @@ __device__ __forceinline__ Words8 ldg256(const void *p) {
     return r;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // Descending order of (score, stride): larger score first, smaller stride index on ties.
 __device__ __forceinline__ bool beats(float xa, int sa, float xb, int sb) { return xa > xb || (xa == xb && sa < sb); }
 
@@ -171,16 +177,26 @@ search_diag(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, in
         cnt = w;
     };
 
-    auto offer = [&](int s, float x) {
-        if (x > v[K - 1]) {
-            lx[32 * cnt] = x;
-            ls[32 * cnt] = s;
+    // Two new scores at a time.  Each one that beats the K-th best so far goes to the list; the sorted
+    // values take both in one pass: with hi >= lo the new j-th best is
+    // max(v[j], min(v[j-1], hi), min(v[j-2], lo)).
+    auto offer2 = [&](int sa, float xa, int sb, float xb) {
+        const float vk = v[K - 1];
+        if (xa > vk) {
+            lx[32 * cnt] = xa;
+            ls[32 * cnt] = sa;
             ++cnt;
         }
-        // sorted insertion of the value: v'[j] = median(v[j-1], x, v[j])
+        if (xb > vk) {
+            lx[32 * cnt] = xb;
+            ls[32 * cnt] = sb;
+            ++cnt;
+        }
+        const float hi = fmaxf(xa, xb), lo = fminf(xa, xb);
 #pragma unroll
-        for (int j = K - 1; j >= 1; --j) v[j] = fmaxf(v[j], fminf(v[j - 1], x));
-        v[0] = fmaxf(v[0], x);
+        for (int j = K - 1; j >= 2; --j) v[j] = max3(v[j], fminf(v[j - 1], hi), fminf(v[j - 2], lo));
+        if (K >= 2) v[1] = max3(v[1], fminf(v[0], hi), lo);
+        v[0] = fmaxf(v[0], hi);
     };
     // scores of one B tile (two strides): two independent accumulation chains, added at the end
     auto score = [&](const Words8 (&kb)[2]) -> float {
@@ -205,8 +221,7 @@ search_diag(const bf16 *__restrict__ q_s, const bf16 *__restrict__ k, Call c, in
             xb = s0 + 2 + u_own < n_own ? xb : -CUDART_INF_F;
         }
         if (__any_sync(0xffffffffu, cnt >= CAP - 1)) compact();   // room for both scores
-        offer(s0 + u_own, xa);
-        offer(s0 + 2 + u_own, xb);
+        offer2(s0 + u_own, xa, s0 + 2 + u_own, xb);
     };
     int s0 = s_min;
     for (; s0 + 4 <= n_all; s0 += 4) step(s0, false);
