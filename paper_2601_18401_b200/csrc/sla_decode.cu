@@ -90,7 +90,9 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
         }
     }
 
-    // ---- the CTA that completes this (batch, KV head) selects and builds the spans
+    // the unsharded step selects in the attention kernel (every CTA for its own head): scores only
+    if (!done) return;
+    // ---- the CTA that completes this (batch, KV head) selects (sequence-sharded step: this rank's candidates)
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -209,13 +211,223 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
 }
 
 // ------------------------------------------------------------------------------------------------
+// Top-k of sc[0..n) by the whole CTA (Section "Span search": TopK over Anchors(i)); sc[x] is the score of
+// stride index s_base + x.  Result in shared memory: sel_anchor[r] / sel_score[r], r = 0 .. top_k - 1, best
+// first (larger score, then the nearer anchor, i.e. the smaller stride index), padded with (-1, -inf).
+//   1. every thread takes the maximum of its contiguous run of scores;
+//   2. warp 0 finds the k-th largest of the 256 thread maxima: at least k scores lie at or above it, so it is a
+//      lower bound of the k-th best score and everything at or above it is a candidate;
+//   3. the candidates are collected (typically a few more than k) and each one's rank among them is its slot.
+// When more candidates turn up than the list holds (many equal scores), every warp selects the k best of its
+// eighth of the scores with the warp routine of the prefill kernels instead, and the 8 k winners are ranked.
+// May overwrite sc.
+struct SelectSmem {
+    static constexpr int kCand = 128;
+    unsigned tmax[kAttnThreads];
+    unsigned thr;
+    int n_cand;
+    unsigned cand_key[kCand];
+    int cand_x[kCand];
+    // fallback
+    float cand_v[kAttnThreads / 32][topk::kCap];
+    int cand_s[kAttnThreads / 32][topk::kCap];
+    int32_t anchor[kAttnThreads / 32][kMaxTopK];
+    float score[kAttnThreads / 32][kMaxTopK];
+};
+
+__device__ inline void cta_select_topk(float *sc, int n, int k, long long i, int s_base, const int *off, SelectSmem &m,
+                                       int *sel_anchor, float *sel_score) {
+    constexpr int kWarps = kAttnThreads / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per_t = (n + kAttnThreads - 1) / kAttnThreads;
+    const int t0 = tid * per_t < n ? tid * per_t : n, t1 = t0 + per_t < n ? t0 + per_t : n;
+    unsigned mx = 0u;   // below every order key of a real score
+    for (int x = t0; x < t1; ++x) mx = max(mx, topk::order_key(sc[x]));
+    m.tmax[tid] = mx;
+    if (tid < k) {
+        sel_anchor[tid] = -1;
+        sel_score[tid] = -CUDART_INF_F;
+    }
+    if (tid == 0) m.n_cand = 0;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = m.tmax[lane * 8 + j];
+        unsigned thr = 0u;
+        for (int r = 0; r < k; ++r) {
+            unsigned best = v[0];
+#pragma unroll
+            for (int j = 1; j < 8; ++j) best = max(best, v[j]);
+            thr = __reduce_max_sync(0xffffffffu, best);
+            if (thr == 0u) break;   // fewer than k threads hold a score: everything is a candidate
+            const unsigned who = __ballot_sync(0xffffffffu, best == thr);
+            if (lane == __ffs(who) - 1) {
+                bool gone = false;   // remove one copy of the maximum
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const bool hit = !gone && v[j] == thr;
+                    v[j] = hit ? 0u : v[j];
+                    gone = gone || hit;
+                }
+            }
+        }
+        if (lane == 0) m.thr = thr;
+    }
+    __syncthreads();
+    const unsigned thr = m.thr;
+    for (int x = t0; x < t1; ++x) {
+        const unsigned key = topk::order_key(sc[x]);
+        if (key >= thr) {
+            const int slot = atomicAdd(&m.n_cand, 1);
+            if (slot < SelectSmem::kCand) {
+                m.cand_key[slot] = key;
+                m.cand_x[slot] = x;
+            }
+        }
+    }
+    __syncthreads();
+    const int nc = m.n_cand;
+    if (nc <= SelectSmem::kCand) {
+        if (tid < nc) {
+            const unsigned kc = m.cand_key[tid];
+            const int xc = m.cand_x[tid];
+            int rank = 0;
+            for (int y = 0; y < nc; ++y) {
+                const unsigned ky = m.cand_key[y];
+                rank += (ky > kc) || (ky == kc && m.cand_x[y] < xc);
+            }
+            if (rank < k) {
+                sel_anchor[rank] = (int)(i + 1 - (off ? (long long)off[s_base + xc] : (long long)(s_base + xc + 1) * (s_base + xc + 1)));
+                sel_score[rank] = sc[xc];
+            }
+        }
+        __syncthreads();
+        return;
+    }
+    // ---- many equal scores: per-warp selection, then the warps' winners ranked
+    const int per = (n + kWarps - 1) / kWarps;
+    const int x0 = warp * per < n ? warp * per : n, x1 = x0 + per < n ? x0 + per : n;
+    topk::select_topk(sc + x0, x1 - x0, k, i, m.cand_v[warp], m.cand_s[warp], m.anchor[warp], m.score[warp], lane,
+                      s_base + x0, off);
+    __syncthreads();
+    for (int e = tid; e < kWarps * k; e += kAttnThreads) {
+        const int w = e / k, j = e % k;
+        const int a = m.anchor[w][j];
+        if (a < 0) continue;
+        const unsigned ka = topk::order_key(m.score[w][j]);
+        int rank = 0;
+        for (int w2 = 0; w2 < kWarps; ++w2)
+            for (int j2 = 0; j2 < k; ++j2) {
+                const int a2 = m.anchor[w2][j2];
+                if (a2 < 0) break;   // a warp's winners come first, its padding last
+                const unsigned k2 = topk::order_key(m.score[w2][j2]);
+                rank += (k2 > ka) || (k2 == ka && a2 > a);
+            }
+        if (rank < k) {
+            sel_anchor[rank] = a;
+            sel_score[rank] = m.score[w][j];
+        }
+    }
+    __syncthreads();
+}
+
+// Span table of one attention unit from the selected anchors (in shared memory: s_anchor[top_k], -1 = none),
+// built by warp 0: piece starts in s_start, cumulative token counts in s_cum, returns the number of pieces.
+// Union mode: the spans of the selected anchors (Algorithm 1: S_t = [max(0,t-b l), min(i,t+f l)]) and the local
+// window W = [max(0, i-w+1), i], sorted by (lo, hi) and clipped to disjoint pieces.  Per-span mode: unit j is
+// J_t of the j-th selected anchor, the part of S_t left of the window and then the window; a head with nothing
+// selected attends to the window alone, carried by its first unit.
+__device__ inline int build_unit_spans(const Call &c, long long i, int j_unit, const int *s_anchor, int *s_lo, int *s_hi,
+                                       int *p_lo, int *p_hi, int *s_start, int *s_cum) {
+    const int lane = threadIdx.x & 31;
+    const long long ell = base_len(c, i);
+    const int n_iv = c.top_k + (c.window > 0 ? 1 : 0);
+    const int w_lo = (int)(i - c.window + 1 > 0 ? i - c.window + 1 : 0);
+    for (int j = lane; j < n_iv; j += 32) {
+        int lo = INT_MAX, hi = -1;
+        if (j == c.top_k) {
+            lo = w_lo;
+            hi = (int)i;
+        } else {
+            const long long t = s_anchor[j];
+            if (t >= 0) {
+                const long long a = t - (long long)c.back * ell, z = t + (long long)c.fwd * ell;
+                lo = (int)(a > 0 ? a : 0);
+                hi = (int)(z < i ? z : i);
+            }
+        }
+        s_lo[j] = lo;
+        s_hi[j] = hi;
+    }
+    __syncwarp();
+    int cnt = 0;
+    if (c.mode == SLA_PER_SPAN) {
+        if (lane == 0) {
+            int n_sel = 0;
+            for (int j = 0; j < c.top_k; ++j) n_sel += s_hi[j] >= 0;
+            const int j = j_unit;
+            int total = 0;
+            s_cum[0] = 0;
+            const bool sel = s_hi[j] >= 0, lone_w = n_sel == 0 && j == 0 && c.window > 0;
+            if (sel) {
+                const int hi_cut = c.window > 0 && s_hi[j] >= w_lo ? w_lo - 1 : s_hi[j];
+                if (s_lo[j] <= hi_cut) {
+                    s_start[cnt] = s_lo[j];
+                    total += hi_cut - s_lo[j] + 1;
+                    s_cum[++cnt] = total;
+                }
+            }
+            if ((sel || lone_w) && c.window > 0) {
+                s_start[cnt] = w_lo;
+                total += (int)i - w_lo + 1;
+                s_cum[++cnt] = total;
+            }
+        }
+        return __shfl_sync(0xffffffffu, cnt, 0);
+    }
+    for (int j = lane; j < n_iv; j += 32) {
+        const int lo = s_lo[j], hi = s_hi[j];
+        int rank = 0;
+        for (int m = 0; m < n_iv; ++m) {
+            const int lm = s_lo[m], hm = s_hi[m];
+            rank += (lm < lo) || (lm == lo && (hm < hi || (hm == hi && m < j)));
+        }
+        p_lo[rank] = lo;
+        p_hi[rank] = hi;
+    }
+    __syncwarp();
+    if (lane == 0) {
+        long long next_free = 0, total = 0;
+        s_cum[0] = 0;
+        for (int a = 0; a < n_iv; ++a) {
+            const int lo = p_lo[a], hi = p_hi[a];
+            if (hi < 0) break;
+            const long long j0 = lo > next_free ? lo : next_free;
+            if (j0 <= hi) {
+                s_start[cnt] = (int)j0;
+                total += hi - j0 + 1;
+                s_cum[cnt + 1] = (int)total;
+                ++cnt;
+            }
+            if ((long long)hi + 1 > next_free) next_free = (long long)hi + 1;
+        }
+    }
+    return __shfl_sync(0xffffffffu, cnt, 0);
+}
+
+// `scores` [B*Hq][n_cand] (the unsharded step): every CTA selects the top-k of its head itself and builds its
+// unit's spans -- nothing waits for a "last" CTA of the scoring kernel; the CTA of split 0 (of the head's first
+// unit) writes the selection out.  `spans` (the sequence-sharded step): the table decode_shard_select built.
 template <typename T, int D>
 __global__ void __launch_bounds__(kAttnThreads)
 decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, Call c,
-            const int *__restrict__ spans, float *__restrict__ partial, int *__restrict__ done,
-            float *__restrict__ unit_out, int *__restrict__ done_head, const int32_t *__restrict__ sel_anchor,
-            const float *__restrict__ sel_score, T *__restrict__ out, float *__restrict__ lse,
+            const int *__restrict__ spans, const float *__restrict__ scores, int n_cand, int s_min,
+            float *__restrict__ partial, int *__restrict__ done,
+            float *__restrict__ unit_out, int *__restrict__ done_head, int32_t *__restrict__ sel_anchor,
+            float *__restrict__ sel_score, T *__restrict__ out, float *__restrict__ lse,
             float *__restrict__ shard_out) {
+    extern __shared__ float s_scores[];   // [n_cand] (unsharded step)
     __shared__ int s_last;
     constexpr int E = Vec16<T>::kElems;
     constexpr int C = 2;                  // 16-byte chunks of a token row per lane: chunks sub and sub + LPR
@@ -224,9 +436,13 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
     constexpr int U = 4;
     constexpr int kWarps = kAttnThreads / 32;
     constexpr int kSlots = kWarps * RPI;  // token rows the CTA reads per load step
+    constexpr int kIv = kMaxTopK + 1;
     __shared__ int s_start[kMaxTopK + 1], s_cum[kMaxTopK + 2];
     __shared__ float s_m[kSlots], s_l[kSlots];
     __shared__ float s_acc[kWarps][D];
+    __shared__ SelectSmem s_sel;
+    __shared__ int s_anchor[kMaxTopK], s_iv[4 * kIv], s_cnt;
+    __shared__ float s_score[kMaxTopK];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sub = lane % LPR, rsel = lane / LPR;
     // attention unit: a head (union mode) or one selected anchor of a head (per-span mode)
@@ -237,13 +453,33 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
     const int n_splits = gridDim.x, split = blockIdx.x;
 
     // launched with programmatic stream serialization: everything above overlaps the tail of the
-    // score kernel, whose results (span table, selected anchors) are read from here on
+    // score kernel, whose results are read from here on
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int *sp = spans + unit * (2 * pcap + 2);
-    const int cnt = sp[2 * pcap + 1];
-    for (int j = tid; j < cnt; j += kAttnThreads) s_start[j] = sp[j];
-    for (int j = tid; j <= cnt; j += kAttnThreads) s_cum[j] = sp[pcap + j];
-    __syncthreads();
+    int cnt;
+    if (scores) {
+        const long long i = c.Lkv - 1;
+        const float *src = scores + bh * n_cand;
+        for (int x = tid; x < n_cand; x += kAttnThreads) s_scores[x] = __ldcg(src + x);
+        __syncthreads();
+        cta_select_topk(s_scores, n_cand, c.top_k, i, s_min, c.off, s_sel, s_anchor, s_score);
+        if (tid < c.top_k && split == 0 && unit % units == 0) {
+            sel_anchor[bh * c.top_k + tid] = s_anchor[tid];
+            sel_score[bh * c.top_k + tid] = s_score[tid];
+        }
+        if (warp == 0) {
+            const int n = build_unit_spans(c, i, (int)(unit % units), s_anchor, s_iv, s_iv + kIv, s_iv + 2 * kIv, s_iv + 3 * kIv,
+                                           s_start, s_cum);
+            if (lane == 0) s_cnt = n;
+        }
+        __syncthreads();
+        cnt = s_cnt;
+    } else {
+        const int *sp = spans + unit * (2 * pcap + 2);
+        cnt = sp[2 * pcap + 1];
+        for (int j = tid; j < cnt; j += kAttnThreads) s_start[j] = sp[j];
+        for (int j = tid; j <= cnt; j += kAttnThreads) s_cum[j] = sp[pcap + j];
+        __syncthreads();
+    }
     const long long total = cnt > 0 ? s_cum[cnt] : 0;
     const long long f_begin = total * split / n_splits, f_end = total * (split + 1) / n_splits;
 
@@ -436,8 +672,8 @@ decode_attn(const T *__restrict__ q, const T *__restrict__ k, const T *__restric
     if (!s_last) return;
     __threadfence();
     if (tid < D) {
-        const int32_t *an = sel_anchor + bh * c.top_k;
-        const float *sc = sel_score + bh * c.top_k;
+        const int *an = s_anchor;      // every CTA of the head holds the head's selection
+        const float *sc = s_score;
         const float *uo = unit_out + bh * units * (D + 2);
         float smax = -CUDART_INF_F;
         int n_sel = 0;
@@ -498,16 +734,12 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
     const int gt = c.G % 8 == 0 ? 8 : c.G % 4 == 0 ? 4 : c.G % 2 == 0 ? 2 : 1;
     dim3 gs(n > 0 ? (n + rows_per_cta - 1) / rows_per_cta : 1, c.B * c.Hkv, c.G / gt);
     const T *qs = (const T *)q_s, *kk = (const T *)k;
-    const size_t smem = (size_t)(kScoreThreads / 32) * (n + 2 * topk::kCap + 4 * (kMaxTopK + 1)) * sizeof(float);
-    if (smem > (size_t)kScoreSmemMax) return cudaErrorInvalidValue;
+    if ((size_t)n * sizeof(float) > 40 * 1024) return cudaErrorInvalidValue;   // the attention kernel holds a head's scores in shared memory
     cudaError_t e = cudaSuccess;
+    // scores only (no completion counter, no shared memory): the attention kernel selects
 #define SLA_LAUNCH_SCORE(GT)                                                                                         \
-    do {                                                                                                             \
-        auto kern = decode_score<T, D, GT>;                                                                          \
-        e = allow_score_smem(kern, smem);                                                                            \
-        if (e == cudaSuccess)                                                                                        \
-            kern<<<gs, kScoreThreads, smem, st>>>(qs, kk, c, n_ctx, n, s_min, scores, done_bg, spans, out_anchor, out_score); \
-    } while (0)
+    decode_score<T, D, GT><<<gs, kScoreThreads, 0, st>>>(qs, kk, c, n_ctx, n, s_min, scores, (int *)nullptr,         \
+                                                          (int *)nullptr, out_anchor, out_score)
     switch (gt) {
         case 8: SLA_LAUNCH_SCORE(8); break;
         case 4: SLA_LAUNCH_SCORE(4); break;
@@ -515,23 +747,22 @@ cudaError_t decode_launch(const void *q_s, const void *q, const void *k, const v
         default: SLA_LAUNCH_SCORE(1); break;
     }
 #undef SLA_LAUNCH_SCORE
-    if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     // programmatic dependent launch: the attention grid is set up while the score kernel drains
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.n_splits, c.B * c.Hq * units);
     cfg.blockDim = dim3(kAttnThreads);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = (size_t)n * sizeof(float);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_attn<T, D>, (const T *)q, kk, (const T *)v, c, (const int *)spans, partial,
-                              done_unit, unit_out, done_head, (const int32_t *)out_anchor, (const float *)out_score,
-                              (T *)out, lse, (float *)nullptr);
+    return cudaLaunchKernelEx(&cfg, decode_attn<T, D>, (const T *)q, kk, (const T *)v, c, (const int *)nullptr,
+                              (const float *)scores, n, s_min, partial, done_unit, unit_out, done_head, out_anchor,
+                              out_score, (T *)out, lse, (float *)nullptr);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -694,8 +925,8 @@ cudaError_t shard_attend_launch(const void *q, const void *k_local, const void *
     if (e != cudaSuccess) return e;
     const T *kk = (const T *)k_local - c.shard_lo * c.kv_st, *vv = (const T *)v_local - c.shard_lo * c.kv_st;
     decode_attn<T, D><<<dim3(p.n_splits, c.B * c.Hq), kAttnThreads, 0, st>>>(
-        (const T *)q, kk, vv, c, spans, partial, done_unit, (float *)nullptr, done_head, out_anchor, out_score,
-        (T *)nullptr, (float *)nullptr, partial_out);
+        (const T *)q, kk, vv, c, spans, (const float *)nullptr, 0, 0, partial, done_unit, (float *)nullptr, done_head,
+        out_anchor, out_score, (T *)nullptr, (float *)nullptr, partial_out);
     return cudaGetLastError();
 }
 
@@ -739,17 +970,19 @@ cudaError_t launch_decode_shard_merge(const float *all_partial, int n_shards, co
 
 
 int decode_attn_blocks_per_sm(int dtype, int D) {
+    // resident CTAs per SM with the shared memory a 16M-token context needs for a head's anchor scores
+    constexpr size_t kOccSmem = 16 * 1024;
     static int cache[2][2] = {{0, 0}, {0, 0}};
     int &slot = cache[dtype == SLA_F32 ? 0 : 1][D == 64 ? 0 : 1];
     if (slot == 0) {
         int n = 0;
         cudaError_t e;
         if (dtype == SLA_F32)
-            e = D == 64 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<float, 64>, kAttnThreads, 0)
-                        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<float, 128>, kAttnThreads, 0);
+            e = D == 64 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<float, 64>, kAttnThreads, kOccSmem)
+                        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<float, 128>, kAttnThreads, kOccSmem);
         else
-            e = D == 64 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<__nv_bfloat16, 64>, kAttnThreads, 0)
-                        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<__nv_bfloat16, 128>, kAttnThreads, 0);
+            e = D == 64 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<__nv_bfloat16, 64>, kAttnThreads, kOccSmem)
+                        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_attn<__nv_bfloat16, 128>, kAttnThreads, kOccSmem);
         slot = (e == cudaSuccess && n > 0) ? n : 1;
     }
     return slot;
