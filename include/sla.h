@@ -278,11 +278,8 @@ sla_status_t sla_decode_step(sla_handle_t handle, const void *q_s, const void *q
  *     1M- and 10M-token configurations with 32 query heads need well under 1 MiB;
  *   - set-up happens inside the call, not at load time: the first call on a device resolves the
  *     array's device address (once per device, with that device current); the first call for each
- *     (device, dtype, head_dim) asks the device for its SM count and the kernel's occupancy; and the
- *     first call on a device whose context is long enough for the scoring kernel to need more than
- *     48 KiB of shared memory (beyond about 1.3 million tokens) raises that kernel's limit, once.  Make
- *     one call per (device, dtype, head_dim), at the longest context you will use, before any stream
- *     capture;
+ *     (device, dtype, head_dim) asks the device for its SM count and the kernel's occupancy.  Make one
+ *     call per (device, dtype, head_dim) before any stream capture;
  *   - all calls on one device share the array: it keeps the previous call's contents (the part that
  *     must start at zero is cleared on the stream at the start of each call), and two calls that
  *     overlap on the GPU -- different streams, or several threads -- race on it.  Serialise them.

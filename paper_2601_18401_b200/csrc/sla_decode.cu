@@ -4,17 +4,20 @@
 // kernel spreads each head's tokens evenly over many CTAs (split-K), streams whole rows with 16-byte
 // loads, keeps a running (max, denominator, numerator) per lane group and merges at the end.
 //
-//   decode_score   grid (anchor chunks, B*Hkv, head tiles)   K anchor rows x G routing queries; the CTA
-//                  that finishes a (batch, KV head) last selects the k best anchors of its G heads,
-//                  builds their spans and clips the overlaps
-//   decode_attn    grid (n_splits, attention units)          online softmax over an even token share;
-//                  the CTA that finishes a unit last merges the split results through their
-//                  log-sum-exp.  Union mode: one unit per head (its spans and the local window, clipped to
-//                  disjoint pieces).  Per-span mode (Algorithm 1 literally): one unit per selected anchor,
-//                  J_t = S_t united with the window; the unit that finishes a head last applies the gate
-//                  of Section "Combination" to the units' outputs
-// "Last" is decided by an atomic counter per (batch, KV head) / per head in the handle's header
-// region; the last CTA puts the counter back to zero, so a step leaves them as it found them.
+//   decode_score   grid (anchor chunks, B*Hkv, head tiles)   K anchor rows x G routing queries -> scores.  In
+//                  the sequence-sharded step the CTA that finishes a (batch, KV head) last also selects this
+//                  rank's k best candidates.
+//   decode_attn    grid (n_splits, attention units)          every CTA first selects the k best anchors of its
+//                  head from the scores (a threshold from the thread maxima, the candidates ranked), builds the
+//                  spans of its unit and clips the overlaps -- redundantly per CTA, so that nothing waits for
+//                  one CTA to do it for all -- then runs the online softmax over an even share of the tokens;
+//                  the CTA that finishes a unit last merges the split results through their log-sum-exp.
+//                  Union mode: one unit per head (its spans and the local window, clipped to disjoint pieces).
+//                  Per-span mode (Algorithm 1 literally): one unit per selected anchor, J_t = S_t united with
+//                  the window; the unit that finishes a head last applies the gate of Section "Combination" to
+//                  the units' outputs.
+// "Last" is decided by an atomic counter per unit / per head in the handle's header region; the last CTA puts
+// the counter back to zero, so a step leaves them as it found them.
 #include <limits.h>
 #include <math_constants.h>
 
