@@ -153,6 +153,19 @@ def test_broadcast_kv_takes_the_generic_kernels(sla, handle):
     assert (lse - lse2).abs().max().item() <= 1e-3
 
 
+def test_prefill_chunks_and_strides_in_groups_of_four(sla, handle):
+    """The search kernel for groups of four query heads on chunks of a longer sequence (query rows that do
+    not start at position 0 or at a multiple of four), on [B,L,H,D] storage, with scales, and the fall
+    back to the 16-anchor kernel for more than 16 slots."""
+    w = workload(n_q_heads=8, n_kv_heads=2, seq_len=2301, span_len=21, top_k=6)
+    run_prefill(sla, handle, w, q_pos0=1111)
+    run_prefill(sla, handle, w, q_pos0=643, Lq=501)
+    run_prefill(sla, handle, w, q_pos0=2300)                  # a single row
+    run_prefill(sla, handle, w, permute=True)
+    run_prefill(sla, handle, w, softmax_scale=0.05, search_scale=-0.5)   # a negative scale reverses the order
+    run_prefill(sla, handle, w.scaled(top_k=20, seq_len=900))
+
+
 def test_tiny_config_full_and_dense(sla, handle):
     """First benchmark configuration in full (fp32, L=4096, l=64): k=4 against the oracle, and
     k=64 (every anchor) against dense causal attention computed here with numpy."""
@@ -305,12 +318,12 @@ def test_error_returns(sla, handle):
     small.close()
 
 
-@pytest.mark.parametrize("seq_len,dtype", [(9000, "bf16"), (12345, "bf16"), (8300, "f32"), (700, "bf16")])
-def test_prefill_host_matches_device_calls(sla, seq_len, dtype):
+@pytest.mark.parametrize("seq_len,dtype,Hq,Hkv", [(9000, "bf16", 4, 2), (12345, "bf16", 8, 2), (8300, "f32", 4, 2), (700, "bf16", 4, 1)])
+def test_prefill_host_matches_device_calls(sla, seq_len, dtype, Hq, Hkv):
     """sla_prefill_host (chunked, copies overlapped with the kernels) against the two device calls on
     the whole sequence and against the oracle: same anchors, outputs within the parity bounds."""
     from paper_2601_18401_b200 import synth
-    w = workload(seq_len=seq_len, dtype=dtype, span_len=24, top_k=5, n_q_heads=4, n_kv_heads=2,
+    w = workload(seq_len=seq_len, dtype=dtype, span_len=24, top_k=5, n_q_heads=Hq, n_kv_heads=Hkv,
                  head_dim=128 if dtype == "bf16" else 64)
     x = synth.make_prefill(w, device="cuda:0")
     params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
