@@ -179,6 +179,15 @@ def attended_pairs(anchor: torch.Tensor, span_len: int, back: int, fwd: int) -> 
     return int(torch.clamp(hi - start + 1, min=0).sum().item())
 
 
+def config_of(w, world: int):
+    """The `config` object of the JSON line: the same for both arms, so that they can be matched."""
+    return {"workload": w.name, "batch_per_gpu": w.batch, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
+            "head_dim": w.head_dim, "seq_len": w.seq_len, "span_len": w.span_len, "top_k": w.top_k,
+            "back_factor": w.back_factor, "fwd_factor": w.fwd_factor, "planted_spans": w.planted_spans,
+            "l2": "inputs (1.3 GB) exceed the 126 MB L2; no flush between steps",
+            "parallelism": f"independent sequences x{world}"}
+
+
 def oracle_sample_rows(L: int, n: int):
     return np.unique(np.linspace(0, L - 1, n).astype(np.int64))
 
@@ -218,8 +227,7 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.batch, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
-                   "head_dim": w.head_dim, "seq_len": w.seq_len, "span_len": w.span_len, "top_k": w.top_k},
+        "config": config_of(w, args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
                          "sample": f"{len(rows)} evenly spaced query positions x all {w.n_q_heads} heads per step"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -502,11 +510,7 @@ def run_ours(args, w):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
-        "config": {"workload": w.name, "batch_per_gpu": B, "q_heads": Hq, "kv_heads": w.n_kv_heads, "head_dim": D,
-                   "seq_len": L, "span_len": w.span_len, "top_k": w.top_k, "back_factor": w.back_factor,
-                   "fwd_factor": w.fwd_factor, "planted_spans": w.planted_spans,
-                   "l2": "inputs (1.3 GB) exceed the 126 MB L2; no flush between steps",
-                   "parallelism": f"independent sequences x{world}"},
+        "config": config_of(w, world),
         "clocks": m["clocks"], "e2e": e2e, "gpu_launches": m["launches"], "roofline": m["roofline"],
         "roofline_search": search_roofline(w, m["search_ms"], probe), "l2_probe": probe,
     }
