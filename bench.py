@@ -38,7 +38,7 @@ METRIC = "prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one tc_attend launch of the default workload
 # (L = 65536): a CONSTANT taken from the one-pass ncu capture of the full-size launch summarised in
-# profiles/bench_prefill_L65536_launch_list.md, not something this run measures
+# the profiles folder, not something this run measures
 TC_ATTEND_DRAM_BYTES_PER_LAUNCH = {65536: 4.74e9, 16384: 0.887e9}
 TRAFFIC_SOURCE = "constant from the one-pass ncu capture summarised under profiles/, not measured by this run"
 NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16, per GPU
