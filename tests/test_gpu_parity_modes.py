@@ -211,3 +211,31 @@ def test_decode_with_general_exponents(sla, handle):
         torch.cuda.synchronize()
         P.check_decode_step(got, synth.to_numpy(x["q_s"]), synth.to_numpy(x["q"]), hk, hv, code, "bf16", n_ctx=n_ctx,
                             top_k=3, span_len=0, back_factor=back, search_exponent=p_search, span_exponent=p_span)
+
+
+def test_pattern_tables_follow_a_change_of_stream(sla):
+    """The handle copies its stride table to the device on the stream of the call that builds it; a call with
+    the same exponent that follows on another stream (no dependency between the streams) must still see
+    the complete table: the library orders the two itself."""
+    from paper_2601_18401_b200 import synth
+    w = workload(span_len=0, top_k=3, seq_len=60000, n_q_heads=4, n_kv_heads=1)
+    x = synth.make_prefill(w, device="cuda:0")
+    params = sla.make_params(3, 0, 3, head_dim=128, search_exponent=1.0 / 3.0, span_exponent=2.0 / 3.0)
+    torch.cuda.synchronize()
+    results = []
+    for rep in range(3):
+        h = sla.Handle(0, 64 << 20)          # a fresh handle: the table is built by the first call
+        s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+        with torch.cuda.stream(s1):
+            a1, v1 = sla.sla_span_search(h, x["q_s"], x["k"], params)
+        with torch.cuda.stream(s2):
+            a2, v2 = sla.sla_span_search(h, x["q_s"], x["k"], params)
+        torch.cuda.synchronize()
+        assert torch.equal(a1, a2) and torch.equal(v1, v2)
+        results.append(a1)
+        h.close()
+    assert torch.equal(results[0], results[1]) and torch.equal(results[0], results[2])
+    host = P.host_inputs(x)
+    rows = np.unique(np.random.default_rng(3).integers(0, w.seq_len, 300))
+    ref = O.span_search(host["q_s"], host["k"], O.BF16, top_k=3, search_exponent=1.0 / 3.0, rows=rows)
+    P.compare_search(results[0], v1, ref, rows=rows, q_s=host["q_s"], k=host["k"], search_exponent=1.0 / 3.0)
