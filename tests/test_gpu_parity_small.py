@@ -164,6 +164,24 @@ def test_prefill_chunks_and_strides_in_groups_of_four(sla, handle):
     run_prefill(sla, handle, w, permute=True)
     run_prefill(sla, handle, w, softmax_scale=0.05, search_scale=-0.5)   # a negative scale reverses the order
     run_prefill(sla, handle, w.scaled(top_k=20, seq_len=900))
+    # tensors that start 16 bytes into a 32-byte line: the 32-byte loads do not apply, the other kernel serves them
+    from paper_2601_18401_b200 import synth
+    x = synth.make_prefill(w, device="cuda:0")
+    off = {}
+    for n, t in x.items():
+        buf = torch.empty(t.numel() + 8, dtype=t.dtype, device=t.device)
+        off[n] = buf[8:].view(t.shape)
+        off[n].copy_(t)
+        assert off[n].data_ptr() % 32 == 16
+    params = sla.make_params(w.top_k, w.span_len, head_dim=w.head_dim)
+    a0, s0 = sla.sla_span_search(handle, x["q_s"], x["k"], params)
+    a1, s1 = sla.sla_span_search(handle, off["q_s"], off["k"], params)
+    torch.cuda.synchronize()
+    same = (a0 == a1).all(-1)
+    assert same.float().mean().item() > 0.999            # two kernels: equal up to near-ties
+    fin = torch.isfinite(s0) & torch.isfinite(s1) & same[..., None]
+    assert torch.equal(torch.isfinite(s0), torch.isfinite(s1))
+    assert (s0 - s1)[fin].abs().max().item() <= 1e-3
 
 
 def test_tiny_config_full_and_dense(sla, handle):
