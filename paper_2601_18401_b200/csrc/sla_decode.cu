@@ -218,8 +218,8 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
 // stride index s_base + x.  Result in shared memory: sel_anchor[r] / sel_score[r], r = 0 .. top_k - 1, best
 // first (larger score, then the nearer anchor, i.e. the smaller stride index), padded with (-1, -inf).
 //   1. every thread takes the maximum of its contiguous run of scores;
-//   2. warp 0 finds the k-th largest of the 256 thread maxima: at least k scores lie at or above it, so it is a
-//      lower bound of the k-th best score and everything at or above it is a candidate;
+//   2. the smallest of the maxima of k (rounded up to a power of two) groups of threads is a lower bound of the
+//      k-th best score -- at least k scores lie at or above it -- and everything at or above it is a candidate;
 //   3. the candidates are collected (typically a few more than k) and each one's rank among them is its slot.
 // When more candidates turn up than the list holds (many equal scores), every warp selects the k best of its
 // eighth of the scores with the warp routine of the prefill kernels instead, and the 8 k winners are ranked.
@@ -227,6 +227,7 @@ decode_score(const T *__restrict__ q_s, const T *__restrict__ k, Call c, long lo
 struct SelectSmem {
     static constexpr int kCand = 128;
     unsigned tmax[kAttnThreads];
+    unsigned gmax[kMaxTopK];
     unsigned thr;
     int n_cand;
     unsigned cand_key[kCand];
@@ -253,29 +254,29 @@ __device__ inline void cta_select_topk(float *sc, int n, int k, long long i, int
     }
     if (tid == 0) m.n_cand = 0;
     __syncthreads();
+    // Threshold: the threads form kp >= k groups (kp the next power of two); every group's maximum is a score
+    // of its own, so at least k scores lie at or above the smallest group maximum: a lower bound of the k-th
+    // best score that costs two short reductions instead of k rounds of a warp-wide maximum.
+    int kp = 1;
+    while (kp < k) kp <<= 1;
+    const int gs = kAttnThreads / kp;   // threads per group (k <= 64: at least 4)
+    if (tid < kp) {
+        unsigned g = 0u;
+        for (int j = 0; j < gs; ++j) g = max(g, m.tmax[tid * gs + j]);
+        m.gmax[tid] = g;
+    }
+    __syncthreads();
     if (warp == 0) {
-        unsigned v[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = m.tmax[lane * 8 + j];
-        unsigned thr = 0u;
-        for (int r = 0; r < k; ++r) {
-            unsigned best = v[0];
-#pragma unroll
-            for (int j = 1; j < 8; ++j) best = max(best, v[j]);
-            thr = __reduce_max_sync(0xffffffffu, best);
-            if (thr == 0u) break;   // fewer than k threads hold a score: everything is a candidate
-            const unsigned who = __ballot_sync(0xffffffffu, best == thr);
-            if (lane == __ffs(who) - 1) {
-                bool gone = false;   // remove one copy of the maximum
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const bool hit = !gone && v[j] == thr;
-                    v[j] = hit ? 0u : v[j];
-                    gone = gone || hit;
-                }
-            }
+        unsigned lo = 0xffffffffu;
+        int filled = 0;
+        for (int j = lane; j < kp; j += 32) {
+            const unsigned g = m.gmax[j];
+            filled += g != 0u;
+            lo = min(lo, g);
         }
-        if (lane == 0) m.thr = thr;
+        lo = __reduce_min_sync(0xffffffffu, lo);
+        filled = __reduce_add_sync(0xffffffffu, filled);
+        if (lane == 0) m.thr = filled >= k ? lo : 0u;   // fewer than k groups hold a score: everything is a candidate
     }
     __syncthreads();
     const unsigned thr = m.thr;
@@ -388,6 +389,46 @@ __device__ inline int build_unit_spans(const Call &c, long long i, int j_unit, c
             }
         }
         return __shfl_sync(0xffffffffu, cnt, 0);
+    }
+    if (n_iv <= 32) {
+        // a lane per interval, everything through shuffles: rank by (lo, hi), then, in sorted order, the running
+        // maximum of the ends before an interval clips its start, a prefix sum of the lengths gives the
+        // cumulative token counts and a ballot the slots of the pieces that are not empty
+        const bool on = lane < n_iv;
+        const int lo = on ? s_lo[lane] : INT_MAX, hi = on ? s_hi[lane] : -1;
+        int rank = 0;
+        for (int m = 0; m < n_iv; ++m) {
+            const int lm = __shfl_sync(0xffffffffu, lo, m), hm = __shfl_sync(0xffffffffu, hi, m);
+            rank += (lm < lo) || (lm == lo && (hm < hi || (hm == hi && m < lane)));
+        }
+        if (on) { p_lo[rank] = lo; p_hi[rank] = hi; }
+        __syncwarp();
+        const int slo = on ? p_lo[lane] : INT_MAX, shi = on ? p_hi[lane] : -1;   // sorted; absent intervals (hi < 0) last
+        // exclusive running maximum of hi + 1 over the intervals before this one
+        int end = shi + 1;   // 0 for an absent interval
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, end, off);
+            if (lane >= off) end = max(end, y);
+        }
+        int prev_end = __shfl_up_sync(0xffffffffu, end, 1);
+        if (lane == 0) prev_end = 0;
+        const int j0 = max(slo, prev_end);
+        const int len = (shi >= 0 && j0 <= shi) ? shi - j0 + 1 : 0;
+        int incl = len;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += y;
+        }
+        const unsigned have = __ballot_sync(0xffffffffu, len > 0);
+        if (len > 0) {
+            const int idx = __popc(have & ((1u << lane) - 1u));
+            s_start[idx] = j0;
+            s_cum[idx + 1] = incl;
+        }
+        if (lane == 0) s_cum[0] = 0;
+        return __popc(have);
     }
     for (int j = lane; j < n_iv; j += 32) {
         const int lo = s_lo[j], hi = s_hi[j];
