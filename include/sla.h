@@ -327,8 +327,8 @@ sla_status_t sla_decode_shard_merge(sla_handle_t handle, int32_t n_shards, const
 
 /* sla_span_search followed by sla_span_attention on HOST buffers (pinned memory gives the best
  * copy rate): copies q_s, q, k, v to the device, runs both steps, copies out, lse, anchors and
- * scores back, and waits for completion.  Sequences of 8192 tokens and more go through in up to
- * sixteen chunks of query positions (chunked prefill: a chunk needs the keys up to its own end), with
+ * scores back, and waits for completion.  Sequences of 4096 tokens and more go through in up to
+ * thirty-two chunks of query positions (chunked prefill: a chunk needs the keys up to its own end), with
  * the copy-in of the next chunk, the kernels of this one and the copy-out of the previous one
  * overlapping on streams the handle owns; results do not depend on the chunking.  Union mode only.
  * All tensors are dense and contiguous

@@ -32,7 +32,7 @@ struct sla_handle_s {
     cudaEvent_t tbl_ev = nullptr;
     cudaStream_t tbl_stream = nullptr;
     // sla_prefill_host: copy-in and copy-out streams and per-chunk events, created on first use
-    static constexpr int kMaxChunks = 16;
+    static constexpr int kMaxChunks = 32;
     cudaStream_t s_in = nullptr, s_out = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_in[kMaxChunks] = {}, ev_done[kMaxChunks] = {};
     char err[256] = {0};
@@ -693,7 +693,7 @@ sla_status_t sla_prefill_host(sla_handle_t h, const void *q_s_host, const void *
     // copy-out of chunk c-1 overlap on three streams.  The device tensors keep the host layout
     // [B, H, L, D]; a chunk of positions is a 2-D copy (one segment per (batch, head)).  Anchors, scores
     // and lse of a chunk are compact [B, Hq, Lc, ...] blocks, as the search call writes them.
-    int n_chunks = (int)(L / 4096);
+    int n_chunks = (int)(L / 2048);
     if (n_chunks > sla_handle_s::kMaxChunks) n_chunks = sla_handle_s::kMaxChunks;
     if (n_chunks < 1) n_chunks = 1;
     const int64_t Lc = ((L + n_chunks - 1) / n_chunks + 127) / 128 * 128;
